@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the SAPS-PSGD gossip round on B200.
+
+One step = one pass of the whole hot path for one round t: peer selection on the host
+(Algorithm 3), then on the GPU the SGD step, the round mask, the emission of the packed
+wire buffer and the pair average (saps_round_pack: a mask-scan kernel and the fused round
+kernel).  Inputs are synthetic Gaussian fp32 matrices of the configured size, resident in
+HBM when the timed region starts.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload vgg16] [--keep-frac 0.01]
+    python bench.py --impl reference ...      # the CPU oracle, as it stands, on the host cores
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "gossip_rounds_per_s"
+UNIT = "rounds/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="vgg16")
+    ap.add_argument("--keep-frac", type=float, default=0.01)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-rounds", type=int, default=4)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock and throttle-reason samples while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(gpu_index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp:
+            f = [v.strip() for v in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands
+# ------------------------------------------------------------------------------------------
+
+def oracle_step(oracle, ps, x, g, w, B, R, t, keep_frac, b_thres, t_thres, cap):
+    """One whole round on the CPU: selection, SGD step, mask, pack, pair average."""
+    import numpy as np
+    pairs, _ = ps.generate_gossip_matrix(B, R, t, b_thres, t_thres)
+    ps.record_round(R, pairs, t)
+    oracle.sgd(x, g, w.lr)
+    m = oracle.mask(w.seed, t, keep_frac, x.shape[1])
+    oracle.pack(x, m, cap)
+    oracle.pair_average(x, np.asarray(pairs, dtype=np.int32), m)
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    import numpy as np
+
+    import oracle
+    from oracle import peer_selection as ps
+    from paper_2002_09692_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    cols = min(w.N, 1 << 21)           # bounded sample: the first `cols` columns of every worker
+    x = synth.gaussian_matrix(w.n, cols, w.x_std, w.seed, 0)
+    g = synth.gaussian_matrix(w.n, cols, w.g_std, w.seed, 1)
+    B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
+    R = ps.new_timestamps(w.n)
+    b_thres, t_thres = ps.default_b_thres(B), ps.default_t_thres(w.n)
+    cap = cols
+    t = 1
+    for _ in range(args.warmup):
+        oracle_step(oracle, ps, x, g, w, B, R, t, args.keep_frac, b_thres, t_thres, cap)
+        t += 1
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(oracle, ps, x, g, w, B, R, t, args.keep_frac, b_thres, t_thres, cap)
+        t += 1
+    dt = time.perf_counter() - t0
+    ms = dt / args.steps * 1e3
+    value = (cols / w.N) / (dt / args.steps)
+    sample = f"first {cols} of {w.N} columns of all {w.n} workers per step; rounds/s scaled by {cols}/{w.N}"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{w.name}: n={w.n}, N={w.N}, keep_frac={args.keep_frac}, adaptive peer selection",
+                   "sample_columns": cols},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import numpy as np
+    import torch
+
+    from paper_2002_09692_b200 import binding as sb
+    from paper_2002_09692_b200 import synth
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    w = synth.WORKLOADS[args.workload]
+    n, N, p = w.n, w.N, args.keep_frac
+    ld = (N + 31) // 32 * 32
+    K, W = args.steps, max(args.warmup, 3)
+
+    # Inputs: Gaussian matrices of the configured standard deviations.  Rank r holds columns
+    # [r N, (r+1) N) of a model with world * N parameters per worker (weak scaling by column
+    # shards: the mask is a function of the global column, the round needs no exchange).
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1000 * w.seed + rank)
+    x = torch.empty(n, ld, dtype=torch.float32, device="cuda")
+    g = torch.empty(n, ld, dtype=torch.float32, device="cuda")
+    x.normal_(0.0, w.x_std, generator=gen)
+    g.normal_(0.0, w.g_std, generator=gen)
+    B = synth.bandwidth_matrix(n, *w.bw_range, seed=w.seed)
+
+    ctx = sb.saps_create_ld(n, N, ld, w.seed)
+    sb.saps_set_column_offset(ctx, rank * N)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.empty(n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.empty(cap, dtype=torch.int32, device="cuda")
+    count = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    stream = torch.cuda.current_stream()
+    ev_k0 = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    ev_k1 = [torch.cuda.Event(enable_timing=True) for _ in range(K)]
+    for e in ev_k0 + ev_k1:
+        e.record(stream)                  # materialises the handles
+    ev_start, ev_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def step(t, k=None):
+        pairs = sb.saps_select_peers(ctx, B, t, n)
+        if k is not None:
+            sb.saps_set_timing_events(ctx, ev_k0[k], ev_k1[k])
+        sb.saps_round_pack(ctx, x, g, w.lr, pairs, t, p, vals, idx, count, stream)
+
+    t = 1
+    for _ in range(W):
+        step(t)
+        t += 1
+    torch.cuda.synchronize()
+    st = sb.saps_status(ctx)
+    if st != 0:
+        raise SystemExit(f"device status after warm-up: {sb.saps_strerror(st)}")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    time.sleep(0.3)
+    barrier()
+    ev_start.record(stream)
+    for k in range(K):
+        step(t, k)
+        t += 1
+    ev_stop.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    sb.saps_set_timing_events(ctx, None, None)
+    st = sb.saps_status(ctx)
+    if st != 0:
+        raise SystemExit(f"device status after the timed region: {sb.saps_strerror(st)}")
+    elapsed_ms = ev_start.elapsed_time(ev_stop)
+    kernel_ms = [a.elapsed_time(b) for a, b in zip(ev_k0, ev_k1)]
+    kept = int(count.cpu().numpy().view(np.uint32)[0])
+    if world > 1:
+        tm = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tm.item())
+
+    ms_per_step = elapsed_ms / K
+    value = world * K / (elapsed_ms * 1e-3)
+    bytes_round = 12.0 * n * N                       # read x, read g, write x
+    bytes_emit = 4.0 * n * kept                      # packed values written by the same pass
+    k_ms = statistics.mean(kernel_ms)
+    achieved = (bytes_round + bytes_emit) / (k_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak_hbm()
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": f"{w.name}: n={n} workers, N={N} fp32 params each (per GPU), keep_frac={p}, "
+                        f"lr={w.lr}, adaptive peer selection on U[{w.bw_range[0]:g},{w.bw_range[1]:g}] Mb/s",
+            "step": "saps_select_peers + saps_round_pack (mask scan kernel + fused SGD/mask/emit/average kernel)",
+            "row_stride": ld, "l2": f"inputs are {2 * 4 * n * N / 1e9:.2f} GB per step, far larger than the 126 MB L2",
+            "sharding": "column shards, one per GPU, no collective" if world > 1 else "single GPU",
+        },
+        "effective_hbm_gbs": bytes_round * K / (elapsed_ms * 1e-3) / 1e9,
+        "frac_of_8tbs": bytes_round * K / (elapsed_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        "kept_columns": kept,
+        "gpu_launches": 2 * K,
+        "clocks": clocks,
+        "roofline": {
+            "bound": "hbm", "kernel": "round_kernel<4,true,true> (fused SGD + mask + emit + pair average)",
+            "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+            "frac": achieved / peak, "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+            "kernel_ms": k_ms, "algorithmic_bytes": bytes_round + bytes_emit, "traffic": None,
+        },
+    }
+
+    if rank == 0 and not args.no_e2e:
+        result["e2e"] = measure_e2e(args, sb, synth, w, ctx, B, t, x, g)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = measure_cpu_baseline(args, synth, w)
+
+    sb.saps_destroy(ctx)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(result))
+
+
+def measure_e2e(args, sb, synth, w, ctx, B, t, x_dev, g_dev):
+    """The same round through the host-buffer entry point: pinned host matrices in, updated
+    model out, copies inside the timed region."""
+    import torch
+    n, N = w.n, w.N
+    hx = torch.empty(n, N, dtype=torch.float32).pin_memory()
+    hg = torch.empty(n, N, dtype=torch.float32).pin_memory()
+    hx.copy_(x_dev[:, :N])
+    hg.copy_(g_dev[:, :N])
+    sb.saps_set_column_offset(ctx, 0)
+    steps = max(1, args.e2e_steps)
+    for _ in range(2):
+        sb.saps_round_host(ctx, hx, hg, w.lr, sb.saps_select_peers(ctx, B, t, n), t, args.keep_frac, x_dev, g_dev)
+        t += 1
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        sb.saps_round_host(ctx, hx, hg, w.lr, sb.saps_select_peers(ctx, B, t, n), t, args.keep_frac, x_dev, g_dev)
+        t += 1
+    dt = time.perf_counter() - t0                     # the call waits for the copies back
+    return {"value": steps / dt, "unit": UNIT, "h2d_bytes_per_step": 2 * 4 * n * N,
+            "d2h_bytes_per_step": 4 * n * N, "ms_per_step": dt / steps * 1e3, "steps": steps,
+            "api": "saps_select_peers + saps_round_host (pinned host x and g in, x out; chunked copy/compute pipeline)"}
+
+
+def measure_cpu_baseline(args, synth, w):
+    """The CPU oracle as it stands (one thread), on a bounded sample of the same workload."""
+    import numpy as np
+
+    import oracle
+    from oracle import peer_selection as ps
+    cols = min(w.N, 1 << 22)
+    x = synth.gaussian_matrix(w.n, cols, w.x_std, w.seed, 0)
+    g = synth.gaussian_matrix(w.n, cols, w.g_std, w.seed, 1)
+    B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
+    R = ps.new_timestamps(w.n)
+    b_thres, t_thres = ps.default_b_thres(B), ps.default_t_thres(w.n)
+    oracle_step(oracle, ps, x, g, w, B, R, 1, args.keep_frac, b_thres, t_thres, cols)
+    rounds = max(1, args.cpu_rounds)
+    t0 = time.perf_counter()
+    for r in range(rounds):
+        oracle_step(oracle, ps, x, g, w, B, R, 2 + r, args.keep_frac, b_thres, t_thres, cols)
+    dt = (time.perf_counter() - t0) / rounds
+    return {"value": (cols / w.N) / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "host_cores_present": os.cpu_count(),
+            "sample": f"{rounds} rounds over the first {cols} of {w.N} columns of all {w.n} workers; "
+                      f"rounds/s scaled by {cols}/{w.N}"}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,217 @@
+/*
+ * saps.h - C ABI of the SAPS-PSGD gossip-round library for NVIDIA B200 (sm_100a).
+ *
+ * The library runs the per-round sparsified pairwise model exchange of SAPS-PSGD
+ * (Tang, Shi, Chu: "Communication-Efficient Decentralized Learning with
+ * Sparsification and Adaptive Peer Selection") for n simulated workers whose
+ * models are the rows of one [n, ld] fp32 matrix in the memory of ONE GPU:
+ *
+ *   1. local SGD step            a_i = x_i - lr * g_i            (Algorithm 2, SGD procedure)
+ *   2. round mask                m_t[k] in {0,1}, Bernoulli(keep_frac), the same for
+ *                                every worker                    (Section II-B, Eq. 3)
+ *   3. pack                      the kept coordinates of every worker, contiguous, in
+ *                                ascending k: the buffer "on the wire"   (Eq. 2, Section II-B)
+ *   4. pair average              kept coordinates of a matched pair (i, j) both become
+ *                                1/2 (a_i + a_j); all others stay a_i
+ *                                                    (Algorithm 2 merge; GenerateW; Eq. 7)
+ *   5. peer selection            the coordinator's bandwidth-aware matching
+ *                                                    (Algorithm 3, GenerateGossipMatrix)
+ *
+ * The paper does not name the generator behind the mask.  This library defines it as a
+ * counter-based hash of (seed, t, k) compared with keep_frac * 2^32 (see saps_round_key).
+ *
+ * Conventions
+ *   - Every function returns an int status (0 = SAPS_OK, negative = error) unless stated;
+ *     nothing throws, aborts or prints.
+ *   - "device" pointers are CUDA device memory owned by the caller; the library neither
+ *     allocates nor frees them.  "host" pointers are ordinary host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All device
+ *     work is enqueued on it and the call returns without waiting.
+ *   - Matrices are row-major fp32, row i = worker i, row stride `ld` elements (ld >= N).
+ *     Elements k >= N of a row are never read or written.
+ *   - n in [1, 64]; N in [1, 2^32 - 1]; t >= 1; keep_frac in [0, 1] (NaN rejected).
+ *   - `pairs` (host, n entries): pairs[i] = peer of worker i, or i when it has none this
+ *     round; it must be an involution (pairs[pairs[i]] == i).
+ *   - fp32 arithmetic is IEEE round-to-nearest, one rounding per operation, never fused:
+ *     a = x - fl(lr * g);  avg = fl(0.5f * fl(a_i + a_j)).  Subnormals are kept.
+ *   - The context owns a small device scratch area (tile states of the compaction scan,
+ *     a status word).  It is allocated by the first call that needs it, on the device that
+ *     is current then; that first call must not happen inside a stream capture.
+ *   - Calls on one context must not overlap on the GPU (use one stream, or order streams
+ *     with events): they share the scratch area.
+ */
+#ifndef SAPS_H_
+#define SAPS_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SAPS_API __attribute__((visibility("default")))
+#else
+#define SAPS_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SAPS_OK            0
+#define SAPS_ERR_INVALID  (-1)  /* bad argument; detected on the host before any launch   */
+#define SAPS_ERR_PAIRS    (-2)  /* pairs is not an involution on 0..n-1                    */
+#define SAPS_ERR_CUDA     (-3)  /* a CUDA runtime call failed (no device, launch error)    */
+#define SAPS_ERR_OVERFLOW (-4)  /* more kept columns than the pack capacity (device-found) */
+#define SAPS_ERR_TIMEOUT  (-5)  /* the compaction scan gave up waiting (device-found)      */
+#define SAPS_ERR_NOMEM    (-6)  /* host or device allocation failed                        */
+
+typedef struct saps_ctx saps_ctx;
+
+/* ---- context ------------------------------------------------------------------------ */
+
+/* Inputs of Algorithms 1-3: n workers, N parameters each, one library seed from which every
+ * round's mask seed s is derived.  Row stride ld = N.  *out receives the context (host
+ * object; no device work happens here). */
+SAPS_API int saps_create(int n, uint64_t N, uint64_t seed, saps_ctx** out);
+
+/* Same, with an explicit row stride ld >= N.  The 128-bit fast path of the round needs
+ * ld % 4 == 0 and 16-byte aligned x and g; any other layout runs a scalar kernel. */
+SAPS_API int saps_create_ld(int n, uint64_t N, uint64_t ld, uint64_t seed, saps_ctx** out);
+
+/* Column sharding (one shard per GPU): this context's column 0 is column col_offset of the
+ * whole model, so that every shard draws its part of the same round mask and a round needs
+ * no exchange between shards.  col_offset + N <= 2^32.  out_idx then holds global columns. */
+SAPS_API int saps_set_column_offset(saps_ctx* ctx, uint64_t col_offset);
+
+/* Frees the context and its device scratch.  Pending work that uses it must have finished. */
+SAPS_API int saps_destroy(saps_ctx* ctx);
+
+/* ---- mask (Section II-B, Eq. 3; Algorithm 2, GenerateRandomMask) ---------------------- */
+
+/* Host only.  The round key (k0, k1) replaces the coordinator's per-round random seed s
+ * (Algorithm 1): a = mix(lo32(seed) ^ 0x243F6A88); a = mix(a ^ hi32(seed));
+ * a = mix(a ^ lo32(t)); a = mix(a ^ hi32(t)); k0 = a; k1 = mix(a ^ 0x85A308D3), with
+ * mix(v): v ^= v>>16; v *= 0x9E3779B9; v ^= v>>15; v *= 0x6A09E667; v ^= v>>16;
+ *         v *= 0xBB67AE85; v ^= v>>15   (uint32, wrapping).
+ * Column k is kept iff H(k) < threshold, where
+ * H(k): v = k ^ k0; v ^= v>>16; v *= 0x9E3779B9; v ^= v>>15; v *= 0x6A09E667; v ^= k1;
+ *       v ^= v>>16; v *= 0xBB67AE85; v ^= v>>15. */
+SAPS_API void saps_round_key(uint64_t seed, uint64_t t, uint32_t* k0, uint32_t* k1);
+
+/* Host only.  floor(keep_frac * 2^32) clamped to [0, 2^32]; 0 for NaN. */
+SAPS_API uint64_t saps_threshold(double keep_frac);
+
+/* Writes the round-t mask as a bitmap: bit (k & 31) of out_bits[k >> 5] is m_t[k]; bits at
+ * and beyond N in the last word are zero.  out_bits: device, ceil(N/32) words. */
+SAPS_API int saps_mask(saps_ctx* ctx, uint64_t t, double keep_frac, uint32_t* out_bits, void* stream);
+
+/* ---- the round (Algorithm 2, SGD procedure and the mask / exchange / merge steps; Eq. 7) - */
+
+/* One fused pass: SGD step, mask, pair average, in place on x.
+ *   x      device [n, ld] fp32, updated in place
+ *   g      device [n, ld] fp32 gradients, or NULL for a round without SGD step (then lr
+ *          must be 0)
+ *   pairs  host, n entries (see above); copied before the call returns
+ * Reads x and g once and writes x once (12 bytes per worker-parameter). */
+SAPS_API int saps_round(saps_ctx* ctx, float* x, const float* g, float lr, const int32_t* pairs,
+               uint64_t t, double keep_frac, void* stream);
+
+/* The same round that also emits the wire buffer of step 3 from the same pass: the packed
+ * values are the post-SGD, pre-average a_i[k] (what worker i sends).  Outputs as saps_pack. */
+SAPS_API int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, const int32_t* pairs,
+                    uint64_t t, double keep_frac, float* out_vals, uint32_t* out_idx,
+                    uint32_t* out_count, void* stream);
+
+/* ---- pack (Eq. 2; "sends the non-zero elements", Section II-B) -------------------------- */
+
+/* Slots per worker that out_vals / out_idx must hold for this keep_frac:
+ * min(N, round_up_32(ceil(N p + 8 sqrt(N p (1-p))) + 64)) with p = threshold / 2^32.
+ * Returns 0 for a NULL context or an invalid keep_frac. */
+SAPS_API uint64_t saps_pack_capacity(const saps_ctx* ctx, double keep_frac);
+
+/* Fixes the capacity to `cap` slots (clamped to N) for every keep_frac, e.g. to a wire
+ * buffer of a given size; 0 restores the formula above.  The paper's "less than N/c" is
+ * loose: the count is Binomial(N, 1/c), so a hard cap can overflow (SAPS_ERR_OVERFLOW). */
+SAPS_API int saps_set_pack_capacity(saps_ctx* ctx, uint64_t cap);
+
+/* Compacts the kept columns of x (as it is now) for every worker.
+ *   out_vals   device [n, cap] fp32, row stride cap = saps_pack_capacity(ctx, keep_frac):
+ *              out_vals[i*cap + r] = x[i][idx[r]]
+ *   out_idx    device [cap] uint32 or NULL: the kept columns in ascending order (one list,
+ *              the mask being the same for every worker)
+ *   out_count  device, one uint32: the number of kept columns
+ * Selection is by mask position, not by value: a kept coordinate equal to 0.0 is sent.
+ * If count > cap, writes stop at cap, out_count still holds the true count and the status
+ * word is set to SAPS_ERR_OVERFLOW.  Slots r >= count are not written. */
+SAPS_API int saps_pack(saps_ctx* ctx, const float* x, uint64_t t, double keep_frac, float* out_vals,
+              uint32_t* out_idx, uint32_t* out_count, void* stream);
+
+/* ---- peer selection (Algorithm 3; GetNewConnectedGraph of Algorithm 1) -------------------- */
+
+/* b_thres: links with min(B_ij, B_ji) >= b_thres form B*.  NaN selects the default, the
+ * median of the symmetrised off-diagonal bandwidths of each call's matrix.
+ * t_thres: an edge is "recently connected" iff R_ij > t - t_thres.  0 selects the default
+ * max(2, 2 ceil(log2 n)). */
+SAPS_API int saps_set_select_params(saps_ctx* ctx, double b_thres, int t_thres);
+
+/* Host only; no device needed.  One run of GenerateGossipMatrix for round t:
+ *   bandwidth  host n x n row-major doubles (symmetrised by min inside; diagonal ignored;
+ *              0 = no link)
+ *   out_pairs  host n entries: the matching as an involution (out_pairs[i] == i only when
+ *              worker i could not be matched: odd n or missing links)
+ * Records the chosen pairs in the context's timestamp matrix R.  t must not decrease
+ * between calls (SAPS_ERR_INVALID).  Any maximum matching of the candidate edges is a
+ * valid answer; which one is returned depends on (seed, t) only. */
+SAPS_API int saps_select_peers(saps_ctx* ctx, const double* bandwidth, uint64_t t, int32_t* out_pairs);
+
+/* Forgets every recorded exchange (R = "never") and the last t. */
+SAPS_API int saps_select_reset(saps_ctx* ctx);
+
+/* Checkpoint / resume of the selection state: R is n x n int64 row-major, INT64_MIN-like
+ * SAPS_NEVER marks "never".  Either pointer may be NULL. */
+#define SAPS_NEVER (-(1LL << 62))
+SAPS_API int saps_get_select_state(const saps_ctx* ctx, int64_t* out_R, uint64_t* out_last_t);
+SAPS_API int saps_set_select_state(saps_ctx* ctx, const int64_t* R, uint64_t last_t);
+
+/* ---- round scheduler (Algorithm 1, the coordinator's loop) --------------------------------- */
+
+/* Enqueues rounds t_first .. t_first + T - 1 on `stream` without any host-device
+ * synchronisation in between.  The matching of each round is
+ *   pairs_list != NULL : pairs_list[r*n .. r*n+n-1] (host, T x n), else
+ *   bandwidth  != NULL : saps_select_peers(ctx, bandwidth, t) (runs on the host ahead of
+ *                        the GPU; it never depends on device data).
+ * out_pairs_log (host, T x n) receives the matchings used, or may be NULL. */
+SAPS_API int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t t_first,
+                    uint64_t T, double keep_frac, const int32_t* pairs_list,
+                    const double* bandwidth, int32_t* out_pairs_log, void* stream);
+
+/* ---- host-buffer entry point ----------------------------------------------------------------- */
+
+/* One round on HOST matrices: copies x_host and g_host ([n, N] fp32, row stride N; pinned
+ * memory recommended) to the device staging buffers, runs the round, copies x back, all in
+ * column chunks pipelined over internal streams, and waits for completion.
+ *   d_x, d_g  device staging, n * ld_dev floats each, ld_dev = N rounded up to a multiple of
+ *             32, 16-byte aligned; caller-owned.  g_host may be NULL (then lr = 0, d_g unused). */
+SAPS_API int saps_round_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
+                    const int32_t* pairs, uint64_t t, double keep_frac, float* d_x, float* d_g);
+
+/* ---- measurement ------------------------------------------------------------------------------- */
+
+/* Optional cudaEvent_t pair (as void*; NULL, NULL switches it off).  When set, saps_round
+ * and saps_round_pack record `before` just ahead of the fused round kernel and `after`
+ * just behind it, on the call's stream, so that a benchmark can time that one kernel inside
+ * a longer step.  The events stay owned by the caller. */
+SAPS_API int saps_set_timing_events(saps_ctx* ctx, void* before, void* after);
+
+/* ---- errors ----------------------------------------------------------------------------------- */
+
+/* Waits for `stream`, then returns in *out_device_status the first error a kernel of this
+ * context recorded since the last call (SAPS_OK, SAPS_ERR_OVERFLOW or SAPS_ERR_TIMEOUT)
+ * and clears it. */
+SAPS_API int saps_status(saps_ctx* ctx, void* stream, int* out_device_status);
+
+/* Static string for a status code. */
+SAPS_API const char* saps_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAPS_H_ */

@@ -1,0 +1,121 @@
+// Internal declarations shared by the translation units of libsaps.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "mask_hash.cuh"
+
+namespace saps {
+
+// One column tile: the unit of the compaction scan and of a round-kernel block.
+constexpr int kTileCols = 2048;
+constexpr int kThreads = 256;
+constexpr uint32_t kMaxWorkers = 64;
+constexpr uint8_t kNoPeer = 0xFF;
+
+// Rows served by one block row of the round kernel: a matched pair (a, b) or a single
+// worker (b == kNoPeer).  Passed by value in the kernel parameter block, so a round needs
+// no host-to-device copy and no staging buffer that a later round could overwrite.
+struct RowGroups {
+    int count;
+    uint8_t a[kMaxWorkers];
+    uint8_t b[kMaxWorkers];
+};
+
+// Device scratch of a context (also the layout of the static no-allocation area).
+//   word 0            status (first device-found error, sticky until read)
+//   word 1            tile ticket of the running scan
+//   words 2..3        unused
+//   then ntiles x u64 tile states {flag << 32 | value}
+//   then ntiles x u32 exclusive prefix of every tile (kept for the fused emission)
+struct ScratchView {
+    int* status;
+    uint32_t* ticket;
+    unsigned long long* tile_state;
+    uint32_t* tile_excl;
+    uint32_t ntiles;
+};
+
+inline size_t scratch_bytes(uint32_t ntiles)
+{
+    return 16 + (size_t)ntiles * 8 + (size_t)ntiles * 4;
+}
+
+inline ScratchView scratch_view(void* base, uint32_t ntiles)
+{
+    char* p = static_cast<char*>(base);
+    ScratchView v;
+    v.status = reinterpret_cast<int*>(p);
+    v.ticket = reinterpret_cast<uint32_t*>(p + 4);
+    v.tile_state = reinterpret_cast<unsigned long long*>(p + 16);
+    v.tile_excl = reinterpret_cast<uint32_t*>(p + 16 + (size_t)ntiles * 8);
+    v.ntiles = ntiles;
+    return v;
+}
+
+// Bytes that must be zero before a scan starts: ticket + padding + tile states.
+inline size_t scratch_clear_bytes(uint32_t ntiles) { return 12 + (size_t)ntiles * 8; }
+
+// Poll budget of the look-back before it gives up (about a second with the back-off used).
+constexpr uint32_t kSpinLimit = 1u << 21;
+
+// ---- launchers (defined in the .cu files) ----------------------------------------------
+
+struct RoundArgs {
+    float* x;
+    const float* g;
+    size_t ld;
+    uint32_t N;
+    float lr;
+    RowGroups groups;
+    RoundKey key;
+    uint32_t col_offset;   // global index of this shard's column 0 (mask hash input)
+    uint32_t tile_begin;   // first column tile to process
+    uint32_t tile_count;   // number of column tiles to process
+    // emission of the wire buffer (all NULL/0 when not emitting)
+    float* out_vals;
+    uint32_t cap;
+    const uint32_t* tile_excl;
+};
+
+cudaError_t launch_round(const RoundArgs& a, bool emit, cudaStream_t stream);
+
+struct PackArgs {
+    const float* x;
+    size_t ld;
+    uint32_t N;
+    int n;
+    RoundKey key;
+    uint32_t col_offset;  // added to k for the hash and in out_idx
+    uint32_t cap;
+    float* out_vals;      // NULL: scan only (indices, count and tile prefixes)
+    uint32_t* out_idx;    // may be NULL
+    uint32_t* out_count;  // may be NULL
+    ScratchView scratch;
+    uint32_t spin_limit;
+};
+
+cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream);
+
+cudaError_t launch_mask(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t* out_bits,
+                        cudaStream_t stream);
+
+// ---- host-side peer selection (select_peers.cpp) ------------------------------------------
+
+struct SelectState {
+    int n = 0;
+    uint64_t seed = 0;
+    double b_thres = 0.0;
+    bool b_thres_default = true;
+    int t_thres = 0;  // 0 = default
+    uint64_t last_t = 0;
+    std::vector<int64_t> R;  // n x n, kNever = never
+};
+
+constexpr int64_t kNever = -(1LL << 62);
+
+int select_peers(SelectState& st, const double* bandwidth, uint64_t t, int32_t* out_pairs);
+
+}  // namespace saps

@@ -1,0 +1,185 @@
+// Compaction of the kept coordinates (x~ = x o m, Eq. 2; the buffer a worker sends,
+// Section II-B) and the mask bitmap.
+//
+// Single pass over column tiles: each warp hashes 32 consecutive columns at a time, a
+// ballot gives their mask word and popc the count; a block scan orders the warps; a
+// decoupled look-back over tile states orders the tiles.  Tiles take their number from an
+// atomic ticket, so every predecessor of a waiting tile is already running or done; the
+// wait is bounded all the same and ends with an error status, never a hang.
+#include "internal.h"
+
+namespace saps {
+namespace {
+
+constexpr unsigned long long kFlagAggregate = 1ull << 32;
+constexpr unsigned long long kFlagInclusive = 2ull << 32;
+
+__device__ __forceinline__ unsigned long long peek_state(const unsigned long long* p)
+{
+    return *reinterpret_cast<const volatile unsigned long long*>(p);
+}
+
+__device__ __forceinline__ uint32_t warp_sum(uint32_t v)
+{
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+    return v;
+}
+
+template <bool GATHER>
+__global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
+{
+    constexpr int kWarps = kThreads / 32;
+    constexpr int kSteps = kTileCols / kThreads;  // ballots per warp
+    __shared__ uint32_t s_tile, s_excl, s_abort;
+    __shared__ uint32_t s_warp_cnt[kWarps];
+    __shared__ uint32_t s_kept[kTileCols];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        s_tile = atomicAdd(a.scratch.ticket, 1u);
+        s_abort = 0;
+    }
+    __syncthreads();
+    const uint32_t tile = s_tile;
+    if (tile >= a.scratch.ntiles) return;  // cannot happen with a cleared ticket; stay in bounds
+
+    // ---- mask words of this warp's 8 x 32 columns ----
+    const uint64_t col_warp = (uint64_t)tile * kTileCols + (uint64_t)warp * (32 * kSteps);
+    uint32_t word[kSteps];
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int s = 0; s < kSteps; ++s) {
+        const uint64_t k = col_warp + s * 32 + lane;
+        const bool kept = (k < a.N) && column_kept(a.col_offset + (uint32_t)k, a.key);
+        word[s] = __ballot_sync(0xFFFFFFFFu, kept);
+        cnt += __popc(word[s]);
+    }
+    if (lane == 0) s_warp_cnt[warp] = cnt;
+    __syncthreads();
+    uint32_t warp_off = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        const uint32_t c = s_warp_cnt[w];
+        warp_off += (w < warp) ? c : 0u;
+        total += c;
+    }
+
+    // ---- order the tiles: decoupled look-back, done by warp 0 ----
+    if (warp == 0) {
+        if (lane == 0)
+            atomicExch(&a.scratch.tile_state[tile],
+                       (tile == 0 ? kFlagInclusive : kFlagAggregate) | total);
+        uint32_t excl = 0;
+        bool ok = true;
+        if (tile > 0) {
+            long long look = (long long)tile - 1;  // newest tile of the window
+            uint32_t polls = 0;
+            while (true) {
+                const long long idx = look - lane;
+                // tiles before the first count as "inclusive prefix 0"
+                const unsigned long long st =
+                    idx >= 0 ? peek_state(&a.scratch.tile_state[idx]) : kFlagInclusive;
+                const uint32_t flag = (uint32_t)(st >> 32);
+                const uint32_t incl = __ballot_sync(0xFFFFFFFFu, flag == 2u);
+                const uint32_t empty = __ballot_sync(0xFFFFFFFFu, flag == 0u);
+                const int first = incl ? (__ffs(incl) - 1) : 32;  // nearest inclusive prefix
+                const uint32_t needed = first >= 31 ? 0xFFFFFFFFu : ((2u << first) - 1u);
+                if (empty & needed) {
+                    // a predecessor has not published yet: back off and poll again
+                    ++polls;
+                    bool give_up = polls > a.spin_limit;
+                    if ((polls & 63u) == 0u)
+                        give_up |= *reinterpret_cast<volatile int*>(a.scratch.status) != 0;
+                    if (__any_sync(0xFFFFFFFFu, give_up)) {
+                        ok = false;
+                        break;
+                    }
+                    __nanosleep(polls < 64u ? 40u : 400u);
+                    continue;
+                }
+                const uint32_t mine = ((needed >> lane) & 1u) ? (uint32_t)st : 0u;
+                excl += warp_sum(mine);
+                if (first < 32) break;
+                look -= 32;
+            }
+        }
+        if (lane == 0) {
+            if (ok) {
+                if (tile > 0) atomicExch(&a.scratch.tile_state[tile], kFlagInclusive | (excl + total));
+                a.scratch.tile_excl[tile] = excl;
+                s_excl = excl;
+            } else {
+                atomicCAS(a.scratch.status, 0, -5 /* SAPS_ERR_TIMEOUT */);
+                s_abort = 1;
+            }
+        }
+    }
+    __syncthreads();
+    if (s_abort) return;
+    const uint32_t base = s_excl;
+
+    // ---- the tile's kept columns, ascending, to shared memory and to out_idx ----
+    uint32_t r = warp_off;
+#pragma unroll
+    for (int s = 0; s < kSteps; ++s) {
+        if ((word[s] >> lane) & 1u) {
+            const uint32_t mine = r + __popc(word[s] & ((1u << lane) - 1u));
+            const uint32_t k = (uint32_t)(col_warp + s * 32 + lane);
+            s_kept[mine] = k;
+            if (a.out_idx != nullptr && base + mine < a.cap) a.out_idx[base + mine] = a.col_offset + k;
+        }
+        r += __popc(word[s]);
+    }
+
+    if (tile == a.scratch.ntiles - 1 && tid == 0) {
+        if (a.out_count != nullptr) *a.out_count = base + total;
+        if (base + total > a.cap) atomicCAS(a.scratch.status, 0, -4 /* SAPS_ERR_OVERFLOW */);
+    }
+
+    // ---- gather: only the kept lanes of x are ever loaded ----
+    if constexpr (GATHER) {
+        __syncthreads();
+        if (total == 0) return;
+        const uint32_t room = base < a.cap ? a.cap - base : 0u;
+        const uint32_t take = total < room ? total : room;
+        for (uint32_t i = 0; i < (uint32_t)a.n; ++i) {
+            const float* __restrict__ row = a.x + (size_t)i * a.ld;
+            float* __restrict__ out = a.out_vals + (size_t)i * a.cap + base;
+            for (uint32_t q = tid; q < take; q += kThreads) out[q] = __ldg(row + s_kept[q]);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) mask_kernel(uint32_t N, uint32_t col_offset, RoundKey key,
+                                                        uint32_t* out_bits)
+{
+    const uint64_t k = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
+    const bool kept = (k < N) && column_kept(col_offset + (uint32_t)k, key);
+    const uint32_t w = __ballot_sync(0xFFFFFFFFu, kept);
+    if ((threadIdx.x & 31) == 0 && k < N) out_bits[k >> 5] = w;
+}
+
+}  // namespace
+
+cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream)
+{
+    const uint32_t ntiles = a.scratch.ntiles;
+    cudaError_t e = cudaMemsetAsync(a.scratch.ticket, 0, scratch_clear_bytes(ntiles), stream);
+    if (e != cudaSuccess) return e;
+    if (a.out_vals != nullptr)
+        pack_kernel<true><<<ntiles, kThreads, 0, stream>>>(a);
+    else
+        pack_kernel<false><<<ntiles, kThreads, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mask(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t* out_bits,
+                        cudaStream_t stream)
+{
+    const uint32_t blocks = (uint32_t)(((uint64_t)N + kThreads - 1) / kThreads);
+    mask_kernel<<<blocks, kThreads, 0, stream>>>(N, col_offset, key, out_bits);
+    return cudaGetLastError();
+}
+
+}  // namespace saps

@@ -1,0 +1,256 @@
+// Fused gossip round: SGD step (Algorithm 2, SGD procedure), round mask (Section II-B,
+// Eq. 3), pair average (Algorithm 2 merge with the weights of GenerateW; Eq. 7), and
+// optionally the emission of the wire buffer (Eq. 2) from the same pass.
+//
+// One block serves one column tile of one row group (a matched pair, or a single worker).
+// Every thread streams 128-bit vectors of x_i, g_i, x_j, g_j, hashes its columns once for
+// both rows, and writes x_i and x_j back: 12 bytes of HBM traffic per worker-parameter,
+// which is what bounds the kernel.  fp32 operations use the round-to-nearest intrinsics so
+// that nothing is contracted into a fused multiply-add.
+#include "internal.h"
+
+namespace saps {
+namespace {
+
+__device__ __forceinline__ float sgd_step(float x, float g, float lr)
+{
+    return __fsub_rn(x, __fmul_rn(lr, g));
+}
+
+__device__ __forceinline__ float pair_mean(float a, float b)
+{
+    return __fmul_rn(0.5f, __fadd_rn(a, b));
+}
+
+template <int VEC>
+struct Chunk {
+    float v[VEC];
+};
+
+// Streaming (evict-first) accesses: every byte is touched once per round.
+template <int VEC>
+__device__ __forceinline__ Chunk<VEC> load_stream(const float* p)
+{
+    Chunk<VEC> c;
+    if constexpr (VEC == 4) {
+        float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+        c.v[0] = t.x; c.v[1] = t.y; c.v[2] = t.z; c.v[3] = t.w;
+    } else {
+        c.v[0] = __ldcs(p);
+    }
+    return c;
+}
+
+template <int VEC>
+__device__ __forceinline__ void store_stream(float* p, const Chunk<VEC>& c)
+{
+    if constexpr (VEC == 4) {
+        __stcs(reinterpret_cast<float4*>(p), make_float4(c.v[0], c.v[1], c.v[2], c.v[3]));
+    } else {
+        __stcs(p, c.v[0]);
+    }
+}
+
+__device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t v, int lane)
+{
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t o = __shfl_up_sync(0xFFFFFFFFu, v, d);
+        if (lane >= d) v += o;
+    }
+    return v;
+}
+
+template <int VEC, bool HAS_G, bool EMIT>
+__global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
+{
+    constexpr int U = kTileCols / (kThreads * VEC);
+    constexpr int kWarps = kThreads / 32;
+    const int tid = threadIdx.x;
+    const uint32_t tile = a.tile_begin + blockIdx.x;
+    const uint32_t ra = a.groups.a[blockIdx.y];
+    const uint32_t rb_raw = a.groups.b[blockIdx.y];
+    const bool paired = rb_raw != kNoPeer;
+    const uint32_t rb = paired ? rb_raw : ra;
+
+    float* __restrict__ xa = a.x + (size_t)ra * a.ld;
+    float* __restrict__ xb = a.x + (size_t)rb * a.ld;
+    const float* __restrict__ ga = HAS_G ? a.g + (size_t)ra * a.ld : nullptr;
+    const float* __restrict__ gb = HAS_G ? a.g + (size_t)rb * a.ld : nullptr;
+
+    // columns reachable by whole vectors; the (N mod 4) leftovers are handled at the end
+    const uint32_t nfull = (VEC == 4) ? (a.N & ~3u) : a.N;
+    const uint64_t col_tile = (uint64_t)tile * kTileCols;
+
+    Chunk<VEC> va[U], vb[U], wa[U], wb[U];
+    bool inb[U];
+    uint32_t col[U];
+
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint64_t k = col_tile + (uint64_t)(u * kThreads + tid) * VEC;
+        inb[u] = k < nfull;
+        col[u] = (uint32_t)k;
+        if (inb[u]) {
+            va[u] = load_stream<VEC>(xa + k);
+            if (HAS_G) wa[u] = load_stream<VEC>(ga + k);
+            if (paired) {
+                vb[u] = load_stream<VEC>(xb + k);
+                if (HAS_G) wb[u] = load_stream<VEC>(gb + k);
+            }
+        }
+    }
+
+    uint32_t bits[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        bits[u] = 0;
+        if (inb[u]) {
+#pragma unroll
+            for (int c = 0; c < VEC; ++c)
+                bits[u] |= (column_kept(a.col_offset + col[u] + c, a.key) ? 1u : 0u) << c;
+            if (HAS_G) {
+#pragma unroll
+                for (int c = 0; c < VEC; ++c) {
+                    va[u].v[c] = sgd_step(va[u].v[c], wa[u].v[c], a.lr);
+                    if (paired) vb[u].v[c] = sgd_step(vb[u].v[c], wb[u].v[c], a.lr);
+                }
+            }
+        }
+    }
+
+    uint32_t rank[U];       // EMIT only: rank of this thread's first kept column
+    uint32_t total = 0;     // EMIT only: kept columns in the vector part of the tile
+    uint32_t excl = 0;
+    if constexpr (EMIT) {
+        __shared__ uint32_t s_warp[U][kWarps];
+        const int lane = tid & 31, warp = tid >> 5;
+        uint32_t within[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t c = __popc(bits[u]);
+            const uint32_t inc = warp_inclusive_sum(c, lane);
+            within[u] = inc - c;
+            if (lane == 31) s_warp[u][warp] = inc;
+        }
+        __syncthreads();
+        excl = a.tile_excl[tile];
+        uint32_t running = excl;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            uint32_t before = 0, all = 0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                const uint32_t s = s_warp[u][w];
+                before += (w < warp) ? s : 0u;
+                all += s;
+            }
+            rank[u] = running + before + within[u];
+            running += all;
+        }
+        total = running - excl;
+        // what each worker sends: its post-SGD value, before the average
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (bits[u]) {
+                uint32_t r = rank[u];
+#pragma unroll
+                for (int c = 0; c < VEC; ++c) {
+                    if ((bits[u] >> c) & 1u) {
+                        if (r < a.cap) {
+                            a.out_vals[(size_t)ra * a.cap + r] = va[u].v[c];
+                            if (paired) a.out_vals[(size_t)rb * a.cap + r] = vb[u].v[c];
+                        }
+                        ++r;
+                    }
+                }
+            }
+        }
+    }
+
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        if (inb[u]) {
+            if (paired) {
+                if (bits[u]) {
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c) {
+                        if ((bits[u] >> c) & 1u) {
+                            const float m = pair_mean(va[u].v[c], vb[u].v[c]);
+                            va[u].v[c] = m;
+                            vb[u].v[c] = m;
+                        }
+                    }
+                }
+                if (HAS_G || bits[u]) {
+                    store_stream<VEC>(xa + col[u], va[u]);
+                    store_stream<VEC>(xb + col[u], vb[u]);
+                }
+            } else if (HAS_G) {
+                store_stream<VEC>(xa + col[u], va[u]);
+            }
+        }
+    }
+
+    // the last (N mod 4) columns of a row, one thread each
+    if constexpr (VEC == 4) {
+        const uint32_t ntail = a.N - nfull;
+        if (ntail != 0 && tid < ntail && col_tile <= nfull && nfull < col_tile + kTileCols) {
+            const uint32_t k = nfull + tid;
+            float pa = xa[k], pb = 0.f;
+            if (HAS_G) pa = sgd_step(pa, ga[k], a.lr);
+            if (paired) {
+                pb = xb[k];
+                if (HAS_G) pb = sgd_step(pb, gb[k], a.lr);
+            }
+            const bool kept = column_kept(a.col_offset + k, a.key);
+            if constexpr (EMIT) {
+                if (kept) {
+                    uint32_t r = excl + total;
+                    for (uint32_t q = nfull; q < k; ++q) r += column_kept(a.col_offset + q, a.key) ? 1u : 0u;
+                    if (r < a.cap) {
+                        a.out_vals[(size_t)ra * a.cap + r] = pa;
+                        if (paired) a.out_vals[(size_t)rb * a.cap + r] = pb;
+                    }
+                }
+            }
+            if (paired) {
+                if (kept) pa = pb = pair_mean(pa, pb);
+                if (HAS_G || kept) {
+                    xa[k] = pa;
+                    xb[k] = pb;
+                }
+            } else if (HAS_G) {
+                xa[k] = pa;
+            }
+        }
+    }
+}
+
+template <int VEC, bool HAS_G, bool EMIT>
+cudaError_t launch_variant(const RoundArgs& a, cudaStream_t stream)
+{
+    dim3 grid(a.tile_count, a.groups.count, 1);
+    round_kernel<VEC, HAS_G, EMIT><<<grid, kThreads, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+template <int VEC>
+cudaError_t launch_vec(const RoundArgs& a, bool emit, cudaStream_t stream)
+{
+    const bool has_g = a.g != nullptr;
+    if (has_g) return emit ? launch_variant<VEC, true, true>(a, stream) : launch_variant<VEC, true, false>(a, stream);
+    return emit ? launch_variant<VEC, false, true>(a, stream) : launch_variant<VEC, false, false>(a, stream);
+}
+
+}  // namespace
+
+cudaError_t launch_round(const RoundArgs& a, bool emit, cudaStream_t stream)
+{
+    if (a.groups.count == 0 || a.tile_count == 0) return cudaSuccess;
+    const bool aligned = (a.ld % 4 == 0) && (reinterpret_cast<uintptr_t>(a.x) % 16 == 0) &&
+                         (a.g == nullptr || reinterpret_cast<uintptr_t>(a.g) % 16 == 0);
+    return aligned ? launch_vec<4>(a, emit, stream) : launch_vec<1>(a, emit, stream);
+}
+
+}  // namespace saps

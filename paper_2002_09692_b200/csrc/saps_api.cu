@@ -1,0 +1,485 @@
+// C ABI of libsaps: context, argument validation, error codes, the round scheduler
+// (Algorithm 1's loop) and the host-buffer entry point.  No device arithmetic lives here.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "../../include/saps.h"
+#include "internal.h"
+
+using namespace saps;
+
+struct saps_ctx {
+    int n;
+    uint64_t N;
+    uint64_t ld;
+    uint64_t seed;
+    uint32_t ntiles;
+    uint64_t col_offset;    // global index of column 0 when this context holds a column shard
+    cudaEvent_t ev_before, ev_after;  // optional: recorded around the round kernel
+    uint64_t cap_override;  // 0 = capacity from the binomial bound
+    // device scratch, allocated on first use on the then-current device
+    void* scratch;
+    int scratch_device;
+    // pipeline of the host-buffer entry point, created on first use
+    static constexpr int kLanes = 3;
+    cudaStream_t lane_stream[kLanes];
+    bool lanes_ready;
+    SelectState select;
+};
+
+namespace {
+
+bool valid_frac(double p) { return p >= 0.0 && p <= 1.0; }  // false for NaN
+
+uint64_t threshold64(double keep_frac)
+{
+    double s = std::floor(keep_frac * 4294967296.0);
+    if (!(s > 0.0)) return 0;
+    if (s >= 4294967296.0) return 1ull << 32;
+    return (uint64_t)s;
+}
+
+RoundKey make_key(uint64_t seed, uint64_t t, double keep_frac)
+{
+    RoundKey key;
+    saps_round_key(seed, t, &key.k0, &key.k1);
+    const uint64_t thr = threshold64(keep_frac);
+    key.all = thr >= (1ull << 32) ? 1u : 0u;
+    key.thr32 = key.all ? 0xFFFFFFFFu : (uint32_t)thr;
+    return key;
+}
+
+int check_pairs(int n, const int32_t* pairs)
+{
+    if (pairs == nullptr) return SAPS_ERR_INVALID;
+    for (int i = 0; i < n; ++i) {
+        const int32_t j = pairs[i];
+        if (j < 0 || j >= n || pairs[j] != i) return SAPS_ERR_PAIRS;
+    }
+    return SAPS_OK;
+}
+
+// Row groups of a round.  A worker without a peer needs a pass only when there is an SGD
+// step to apply or a wire buffer to emit.
+RowGroups make_groups(int n, const int32_t* pairs, bool singles)
+{
+    RowGroups rg;
+    rg.count = 0;
+    for (int i = 0; i < n; ++i) {
+        const int j = pairs[i];
+        if (j > i) {
+            rg.a[rg.count] = (uint8_t)i;
+            rg.b[rg.count] = (uint8_t)j;
+            ++rg.count;
+        } else if (j == i && singles) {
+            rg.a[rg.count] = (uint8_t)i;
+            rg.b[rg.count] = kNoPeer;
+            ++rg.count;
+        }
+    }
+    return rg;
+}
+
+int ensure_scratch(saps_ctx* ctx)
+{
+    if (ctx->scratch != nullptr) return SAPS_OK;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return SAPS_ERR_CUDA;
+    }
+    void* p = nullptr;
+    const size_t bytes = scratch_bytes(ctx->ntiles);
+    if (cudaMalloc(&p, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return SAPS_ERR_NOMEM;
+    }
+    if (cudaMemset(p, 0, bytes) != cudaSuccess) {
+        cudaFree(p);
+        cudaGetLastError();
+        return SAPS_ERR_CUDA;
+    }
+    ctx->scratch = p;
+    ctx->scratch_device = dev;
+    return SAPS_OK;
+}
+
+int check_round_args(const saps_ctx* ctx, const float* x, const float* g, float lr, uint64_t t,
+                     double keep_frac)
+{
+    if (ctx == nullptr || x == nullptr || t == 0 || !valid_frac(keep_frac)) return SAPS_ERR_INVALID;
+    if (g == nullptr && lr != 0.0f) return SAPS_ERR_INVALID;
+    if (lr != lr) return SAPS_ERR_INVALID;
+    return SAPS_OK;
+}
+
+RoundArgs round_args(const saps_ctx* ctx, float* x, const float* g, float lr, const RowGroups& rg,
+                     const RoundKey& key, uint64_t ld = 0)
+{
+    RoundArgs a;
+    a.x = x;
+    a.g = g;
+    a.ld = (size_t)(ld ? ld : ctx->ld);
+    a.N = (uint32_t)ctx->N;
+    a.lr = lr;
+    a.groups = rg;
+    a.key = key;
+    a.col_offset = (uint32_t)ctx->col_offset;
+    a.tile_begin = 0;
+    a.tile_count = ctx->ntiles;
+    a.out_vals = nullptr;
+    a.cap = 0;
+    a.tile_excl = nullptr;
+    return a;
+}
+
+// Launch of the round kernel, bracketed by the caller's timing events when they are set.
+int timed_round(const saps_ctx* ctx, const RoundArgs& a, bool emit, cudaStream_t stream)
+{
+    if (ctx->ev_before != nullptr && cudaEventRecord(ctx->ev_before, stream) != cudaSuccess) return SAPS_ERR_CUDA;
+    if (launch_round(a, emit, stream) != cudaSuccess) return SAPS_ERR_CUDA;
+    if (ctx->ev_after != nullptr && cudaEventRecord(ctx->ev_after, stream) != cudaSuccess) return SAPS_ERR_CUDA;
+    return SAPS_OK;
+}
+
+uint64_t capacity_for(uint64_t N, double keep_frac)
+{
+    const double p = (double)threshold64(keep_frac) / 4294967296.0;
+    const double mean = (double)N * p;
+    const double sd = std::sqrt((double)N * p * (1.0 - p));
+    uint64_t c = (uint64_t)std::ceil(mean + 8.0 * sd) + 64;
+    c = (c + 31) / 32 * 32;
+    return c < N ? c : N;
+}
+
+}  // namespace
+
+extern "C" {
+
+int saps_create_ld(int n, uint64_t N, uint64_t ld, uint64_t seed, saps_ctx** out)
+{
+    if (out == nullptr) return SAPS_ERR_INVALID;
+    *out = nullptr;
+    if (n < 1 || n > (int)kMaxWorkers || N < 1 || N > 0xFFFFFFFFull || ld < N) return SAPS_ERR_INVALID;
+    saps_ctx* ctx = new (std::nothrow) saps_ctx();
+    if (ctx == nullptr) return SAPS_ERR_NOMEM;
+    ctx->n = n;
+    ctx->N = N;
+    ctx->ld = ld;
+    ctx->seed = seed;
+    ctx->ntiles = (uint32_t)((N + kTileCols - 1) / kTileCols);
+    ctx->cap_override = 0;
+    ctx->ev_before = nullptr;
+    ctx->ev_after = nullptr;
+    ctx->col_offset = 0;
+    ctx->scratch = nullptr;
+    ctx->scratch_device = -1;
+    ctx->lanes_ready = false;
+    ctx->select.n = n;
+    ctx->select.seed = seed;
+    try {
+        ctx->select.R.assign((size_t)n * n, kNever);
+    } catch (...) {
+        delete ctx;
+        return SAPS_ERR_NOMEM;
+    }
+    *out = ctx;
+    return SAPS_OK;
+}
+
+int saps_create(int n, uint64_t N, uint64_t seed, saps_ctx** out)
+{
+    return saps_create_ld(n, N, N, seed, out);
+}
+
+int saps_destroy(saps_ctx* ctx)
+{
+    if (ctx == nullptr) return SAPS_ERR_INVALID;
+    if (ctx->lanes_ready)
+        for (int l = 0; l < saps_ctx::kLanes; ++l) cudaStreamDestroy(ctx->lane_stream[l]);
+    if (ctx->scratch != nullptr) cudaFree(ctx->scratch);
+    delete ctx;
+    return SAPS_OK;
+}
+
+void saps_round_key(uint64_t seed, uint64_t t, uint32_t* k0, uint32_t* k1)
+{
+    uint32_t a = mix32((uint32_t)(seed & 0xFFFFFFFFull) ^ kSeedPad);
+    a = mix32(a ^ (uint32_t)(seed >> 32));
+    a = mix32(a ^ (uint32_t)(t & 0xFFFFFFFFull));
+    a = mix32(a ^ (uint32_t)(t >> 32));
+    if (k0) *k0 = a;
+    if (k1) *k1 = mix32(a ^ kKeyPad);
+}
+
+uint64_t saps_threshold(double keep_frac) { return threshold64(keep_frac); }
+
+int saps_mask(saps_ctx* ctx, uint64_t t, double keep_frac, uint32_t* out_bits, void* stream)
+{
+    if (ctx == nullptr || out_bits == nullptr || t == 0 || !valid_frac(keep_frac)) return SAPS_ERR_INVALID;
+    const RoundKey key = make_key(ctx->seed, t, keep_frac);
+    return launch_mask((uint32_t)ctx->N, (uint32_t)ctx->col_offset, key, out_bits, (cudaStream_t)stream) == cudaSuccess ? SAPS_OK
+                                                                                              : SAPS_ERR_CUDA;
+}
+
+int saps_round(saps_ctx* ctx, float* x, const float* g, float lr, const int32_t* pairs, uint64_t t,
+               double keep_frac, void* stream)
+{
+    int rc = check_round_args(ctx, x, g, lr, t, keep_frac);
+    if (rc != SAPS_OK) return rc;
+    rc = check_pairs(ctx->n, pairs);
+    if (rc != SAPS_OK) return rc;
+    const RowGroups rg = make_groups(ctx->n, pairs, g != nullptr);
+    const RoundArgs a = round_args(ctx, x, g, lr, rg, make_key(ctx->seed, t, keep_frac));
+    return timed_round(ctx, a, false, (cudaStream_t)stream);
+}
+
+uint64_t saps_pack_capacity(const saps_ctx* ctx, double keep_frac)
+{
+    if (ctx == nullptr || !valid_frac(keep_frac)) return 0;
+    if (ctx->cap_override != 0) return ctx->cap_override < ctx->N ? ctx->cap_override : ctx->N;
+    return capacity_for(ctx->N, keep_frac);
+}
+
+int saps_set_column_offset(saps_ctx* ctx, uint64_t col_offset)
+{
+    if (ctx == nullptr || col_offset + ctx->N > (1ull << 32)) return SAPS_ERR_INVALID;
+    ctx->col_offset = col_offset;
+    return SAPS_OK;
+}
+
+int saps_set_timing_events(saps_ctx* ctx, void* before, void* after)
+{
+    if (ctx == nullptr) return SAPS_ERR_INVALID;
+    ctx->ev_before = (cudaEvent_t)before;
+    ctx->ev_after = (cudaEvent_t)after;
+    return SAPS_OK;
+}
+
+int saps_set_pack_capacity(saps_ctx* ctx, uint64_t cap)
+{
+    if (ctx == nullptr || cap > 0xFFFFFFFFull) return SAPS_ERR_INVALID;
+    ctx->cap_override = cap;
+    return SAPS_OK;
+}
+
+int saps_pack(saps_ctx* ctx, const float* x, uint64_t t, double keep_frac, float* out_vals,
+              uint32_t* out_idx, uint32_t* out_count, void* stream)
+{
+    if (ctx == nullptr || x == nullptr || out_vals == nullptr || out_count == nullptr || t == 0 ||
+        !valid_frac(keep_frac))
+        return SAPS_ERR_INVALID;
+    int rc = ensure_scratch(ctx);
+    if (rc != SAPS_OK) return rc;
+    PackArgs a;
+    a.x = x;
+    a.ld = (size_t)ctx->ld;
+    a.N = (uint32_t)ctx->N;
+    a.n = ctx->n;
+    a.key = make_key(ctx->seed, t, keep_frac);
+    a.col_offset = (uint32_t)ctx->col_offset;
+    a.cap = (uint32_t)saps_pack_capacity(ctx, keep_frac);
+    a.out_vals = out_vals;
+    a.out_idx = out_idx;
+    a.out_count = out_count;
+    a.scratch = scratch_view(ctx->scratch, ctx->ntiles);
+    a.spin_limit = kSpinLimit;
+    return launch_pack(a, (cudaStream_t)stream) == cudaSuccess ? SAPS_OK : SAPS_ERR_CUDA;
+}
+
+int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, const int32_t* pairs,
+                    uint64_t t, double keep_frac, float* out_vals, uint32_t* out_idx,
+                    uint32_t* out_count, void* stream)
+{
+    int rc = check_round_args(ctx, x, g, lr, t, keep_frac);
+    if (rc != SAPS_OK) return rc;
+    if (out_vals == nullptr || out_count == nullptr) return SAPS_ERR_INVALID;
+    rc = check_pairs(ctx->n, pairs);
+    if (rc != SAPS_OK) return rc;
+    rc = ensure_scratch(ctx);
+    if (rc != SAPS_OK) return rc;
+    const RoundKey key = make_key(ctx->seed, t, keep_frac);
+    const uint32_t cap = (uint32_t)saps_pack_capacity(ctx, keep_frac);
+    // pass 1 touches no model data: mask scan -> indices, count and per-tile prefixes
+    PackArgs p;
+    p.x = nullptr;
+    p.ld = (size_t)ctx->ld;
+    p.N = (uint32_t)ctx->N;
+    p.n = ctx->n;
+    p.key = key;
+    p.col_offset = (uint32_t)ctx->col_offset;
+    p.cap = cap;
+    p.out_vals = nullptr;
+    p.out_idx = out_idx;
+    p.out_count = out_count;
+    p.scratch = scratch_view(ctx->scratch, ctx->ntiles);
+    p.spin_limit = kSpinLimit;
+    if (launch_pack(p, (cudaStream_t)stream) != cudaSuccess) return SAPS_ERR_CUDA;
+    // pass 2: the fused round writes each worker's kept values at the scanned ranks
+    const RowGroups rg = make_groups(ctx->n, pairs, true);
+    RoundArgs a = round_args(ctx, x, g, lr, rg, key);
+    a.out_vals = out_vals;
+    a.cap = cap;
+    a.tile_excl = p.scratch.tile_excl;
+    return timed_round(ctx, a, true, (cudaStream_t)stream);
+}
+
+int saps_set_select_params(saps_ctx* ctx, double b_thres, int t_thres)
+{
+    if (ctx == nullptr || t_thres < 0) return SAPS_ERR_INVALID;
+    ctx->select.b_thres_default = b_thres != b_thres;
+    ctx->select.b_thres = ctx->select.b_thres_default ? 0.0 : b_thres;
+    ctx->select.t_thres = t_thres;
+    return SAPS_OK;
+}
+
+int saps_select_peers(saps_ctx* ctx, const double* bandwidth, uint64_t t, int32_t* out_pairs)
+{
+    if (ctx == nullptr || bandwidth == nullptr || out_pairs == nullptr || t == 0) return SAPS_ERR_INVALID;
+    return select_peers(ctx->select, bandwidth, t, out_pairs);
+}
+
+int saps_select_reset(saps_ctx* ctx)
+{
+    if (ctx == nullptr) return SAPS_ERR_INVALID;
+    ctx->select.R.assign(ctx->select.R.size(), kNever);
+    ctx->select.last_t = 0;
+    return SAPS_OK;
+}
+
+int saps_get_select_state(const saps_ctx* ctx, int64_t* out_R, uint64_t* out_last_t)
+{
+    if (ctx == nullptr) return SAPS_ERR_INVALID;
+    if (out_R) std::memcpy(out_R, ctx->select.R.data(), ctx->select.R.size() * sizeof(int64_t));
+    if (out_last_t) *out_last_t = ctx->select.last_t;
+    return SAPS_OK;
+}
+
+int saps_set_select_state(saps_ctx* ctx, const int64_t* R, uint64_t last_t)
+{
+    if (ctx == nullptr) return SAPS_ERR_INVALID;
+    if (R) std::memcpy(ctx->select.R.data(), R, ctx->select.R.size() * sizeof(int64_t));
+    ctx->select.last_t = last_t;
+    return SAPS_OK;
+}
+
+int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t t_first, uint64_t T,
+                    double keep_frac, const int32_t* pairs_list, const double* bandwidth,
+                    int32_t* out_pairs_log, void* stream)
+{
+    int rc = check_round_args(ctx, x, g, lr, t_first, keep_frac);
+    if (rc != SAPS_OK) return rc;
+    if (pairs_list == nullptr && bandwidth == nullptr) return SAPS_ERR_INVALID;
+    const int n = ctx->n;
+    int32_t chosen[kMaxWorkers];
+    for (uint64_t r = 0; r < T; ++r) {
+        const uint64_t t = t_first + r;
+        const int32_t* pairs;
+        if (pairs_list != nullptr) {
+            pairs = pairs_list + r * (uint64_t)n;
+        } else {
+            rc = select_peers(ctx->select, bandwidth, t, chosen);
+            if (rc != SAPS_OK) return rc;
+            pairs = chosen;
+        }
+        rc = check_pairs(n, pairs);
+        if (rc != SAPS_OK) return rc;
+        if (out_pairs_log != nullptr) std::memcpy(out_pairs_log + r * (uint64_t)n, pairs, sizeof(int32_t) * n);
+        const RowGroups rg = make_groups(n, pairs, g != nullptr);
+        const RoundArgs a = round_args(ctx, x, g, lr, rg, make_key(ctx->seed, t, keep_frac));
+        if (launch_round(a, false, (cudaStream_t)stream) != cudaSuccess) return SAPS_ERR_CUDA;
+    }
+    return SAPS_OK;
+}
+
+int saps_round_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr, const int32_t* pairs,
+                    uint64_t t, double keep_frac, float* d_x, float* d_g)
+{
+    int rc = check_round_args(ctx, x_host, g_host, lr, t, keep_frac);
+    if (rc != SAPS_OK) return rc;
+    if (d_x == nullptr || (g_host != nullptr && d_g == nullptr)) return SAPS_ERR_INVALID;
+    rc = check_pairs(ctx->n, pairs);
+    if (rc != SAPS_OK) return rc;
+    if (!ctx->lanes_ready) {
+        for (int l = 0; l < saps_ctx::kLanes; ++l) {
+            if (cudaStreamCreateWithFlags(&ctx->lane_stream[l], cudaStreamNonBlocking) != cudaSuccess) {
+                for (int m = 0; m < l; ++m) cudaStreamDestroy(ctx->lane_stream[m]);
+                cudaGetLastError();
+                return SAPS_ERR_CUDA;
+            }
+        }
+        ctx->lanes_ready = true;
+    }
+    const int n = ctx->n;
+    const uint64_t N = ctx->N;
+    const uint64_t ld_dev = (N + 31) / 32 * 32;
+    // The round acts column by column, so column chunks are independent: copy in, compute
+    // and copy out chunk by chunk, round-robin over a few streams, so that the two copy
+    // directions and the kernel overlap.
+    const RowGroups rg = make_groups(n, pairs, g_host != nullptr);
+    const RoundKey key = make_key(ctx->seed, t, keep_frac);
+    const uint32_t tiles_per_chunk = 512;  // 1 Mi columns: n x 4 MiB per matrix and chunk
+    bool failed = false;
+    int lane = 0;
+    for (uint32_t tb = 0; tb < ctx->ntiles && !failed; tb += tiles_per_chunk, lane = (lane + 1) % saps_ctx::kLanes) {
+        const uint32_t tc = ctx->ntiles - tb < tiles_per_chunk ? ctx->ntiles - tb : tiles_per_chunk;
+        const uint64_t c0 = (uint64_t)tb * kTileCols;
+        const uint64_t c1 = c0 + (uint64_t)tc * kTileCols < N ? c0 + (uint64_t)tc * kTileCols : N;
+        const size_t width = (size_t)(c1 - c0) * sizeof(float);
+        cudaStream_t s = ctx->lane_stream[lane];
+        failed |= cudaMemcpy2DAsync(d_x + c0, ld_dev * sizeof(float), x_host + c0, N * sizeof(float), width, n,
+                                    cudaMemcpyHostToDevice, s) != cudaSuccess;
+        if (g_host != nullptr)
+            failed |= cudaMemcpy2DAsync(d_g + c0, ld_dev * sizeof(float), g_host + c0, N * sizeof(float), width,
+                                        n, cudaMemcpyHostToDevice, s) != cudaSuccess;
+        RoundArgs a = round_args(ctx, d_x, g_host != nullptr ? d_g : nullptr, lr, rg, key, ld_dev);
+        a.tile_begin = tb;
+        a.tile_count = tc;
+        failed |= launch_round(a, false, s) != cudaSuccess;
+        failed |= cudaMemcpy2DAsync(x_host + c0, N * sizeof(float), d_x + c0, ld_dev * sizeof(float), width, n,
+                                    cudaMemcpyDeviceToHost, s) != cudaSuccess;
+    }
+    for (int l = 0; l < saps_ctx::kLanes; ++l) failed |= cudaStreamSynchronize(ctx->lane_stream[l]) != cudaSuccess;
+    if (failed) {
+        cudaGetLastError();
+        return SAPS_ERR_CUDA;
+    }
+    return SAPS_OK;
+}
+
+int saps_status(saps_ctx* ctx, void* stream, int* out_device_status)
+{
+    if (ctx == nullptr || out_device_status == nullptr) return SAPS_ERR_INVALID;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SAPS_ERR_CUDA;
+    }
+    *out_device_status = SAPS_OK;
+    if (ctx->scratch == nullptr) return SAPS_OK;
+    int st = 0;
+    if (cudaMemcpy(&st, ctx->scratch, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess ||
+        (st != 0 && cudaMemset(ctx->scratch, 0, sizeof(int)) != cudaSuccess)) {
+        cudaGetLastError();
+        return SAPS_ERR_CUDA;
+    }
+    *out_device_status = st;
+    return SAPS_OK;
+}
+
+const char* saps_strerror(int status)
+{
+    switch (status) {
+        case SAPS_OK: return "ok";
+        case SAPS_ERR_INVALID: return "invalid argument";
+        case SAPS_ERR_PAIRS: return "pairs is not an involution on 0..n-1";
+        case SAPS_ERR_CUDA: return "CUDA runtime call failed";
+        case SAPS_ERR_OVERFLOW: return "more kept columns than the pack capacity";
+        case SAPS_ERR_TIMEOUT: return "compaction scan gave up waiting for a predecessor tile";
+        case SAPS_ERR_NOMEM: return "out of memory";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,254 @@
+// Host-side peer selection: GenerateGossipMatrix (Algorithm 3) with GetNewConnectedGraph
+// (Algorithm 1).  n <= 64, so this is control code that runs on the host ahead of the GPU.
+//
+// Choices where the paper leaves room:
+//   B symmetrised by min (Section II-C); B*_ij = [B_ij >= B_thres]; an edge is recent iff
+//   R_ij > t - T_thres and "never" is not recent; a disconnected recent graph yields every
+//   cross-component link with B_ij > 0; leftovers are paired over every link with B_ij > 0;
+//   the matching is maximum-cardinality (Edmonds' blossom algorithm), started "randomly from
+//   different nodes" by relabelling the vertices with a (seed, t, stage)-keyed shuffle.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+#include "../../include/saps.h"
+#include "internal.h"
+
+namespace saps {
+namespace {
+
+// Maximum-cardinality matching in a general graph: breadth-first alternating trees with
+// blossoms kept contracted through a "base" label per vertex.
+class BlossomMatcher {
+public:
+    BlossomMatcher(int n, const std::vector<uint8_t>& adj)
+        : n_(n), adj_(adj), mate_(n, -1), up_(n), base_(n), seen_(n), in_blossom_(n), fifo_(n) {}
+
+    const std::vector<int>& solve()
+    {
+        for (int v = 0; v < n_; ++v) {
+            if (mate_[v] != -1) continue;
+            const int leaf = grow_tree(v);
+            // flip the alternating path leaf -> root
+            for (int w = leaf; w != -1;) {
+                const int pv = up_[w];
+                const int next = mate_[pv];
+                mate_[w] = pv;
+                mate_[pv] = w;
+                w = next;
+            }
+        }
+        return mate_;
+    }
+
+private:
+    bool edge(int a, int b) const { return adj_[(size_t)a * n_ + b] != 0; }
+
+    // first common blossom base on the two root paths
+    int common_base(int a, int b)
+    {
+        std::vector<char> on_path(n_, 0);
+        for (int v = a;;) {
+            v = base_[v];
+            on_path[v] = 1;
+            if (mate_[v] == -1) break;
+            v = up_[mate_[v]];
+        }
+        for (int v = b;;) {
+            v = base_[v];
+            if (on_path[v]) return v;
+            v = up_[mate_[v]];
+        }
+    }
+
+    // walk from v down to the blossom base b, marking the bases on the way and re-hanging
+    // the odd vertices so that the path can later be flipped in either direction
+    void mark_side(int v, int b, int child)
+    {
+        while (base_[v] != b) {
+            in_blossom_[base_[v]] = 1;
+            in_blossom_[base_[mate_[v]]] = 1;
+            up_[v] = child;
+            child = mate_[v];
+            v = up_[mate_[v]];
+        }
+    }
+
+    // returns the free vertex that ends an augmenting path from root, or -1
+    int grow_tree(int root)
+    {
+        std::fill(seen_.begin(), seen_.end(), 0);
+        std::fill(up_.begin(), up_.end(), -1);
+        for (int i = 0; i < n_; ++i) base_[i] = i;
+        int head = 0, tail = 0;
+        fifo_[tail++] = root;
+        seen_[root] = 1;
+        while (head < tail) {
+            const int v = fifo_[head++];
+            for (int w = 0; w < n_; ++w) {
+                if (!edge(v, w) || base_[v] == base_[w] || mate_[v] == w) continue;
+                if (w == root || (mate_[w] != -1 && up_[mate_[w]] != -1)) {
+                    // w is an even vertex of the tree: odd cycle, contract it
+                    const int b = common_base(v, w);
+                    std::fill(in_blossom_.begin(), in_blossom_.end(), 0);
+                    mark_side(v, b, w);
+                    mark_side(w, b, v);
+                    for (int i = 0; i < n_; ++i) {
+                        if (!in_blossom_[base_[i]]) continue;
+                        base_[i] = b;
+                        if (!seen_[i]) {
+                            seen_[i] = 1;
+                            fifo_[tail++] = i;
+                        }
+                    }
+                } else if (up_[w] == -1) {
+                    up_[w] = v;
+                    if (mate_[w] == -1) return w;
+                    seen_[mate_[w]] = 1;
+                    fifo_[tail++] = mate_[w];
+                }
+            }
+        }
+        return -1;
+    }
+
+    int n_;
+    const std::vector<uint8_t>& adj_;
+    std::vector<int> mate_, up_, base_;
+    std::vector<char> seen_, in_blossom_;
+    std::vector<int> fifo_;
+};
+
+// RandomlyMaxMatch: relabel the vertices by a keyed shuffle, match, map back.
+// Returns the number of matched pairs; mate[v] = partner or -1.
+int randomly_max_match(int n, const std::vector<uint8_t>& E, uint64_t seed, uint64_t t, uint32_t stage,
+                       std::vector<int>& mate)
+{
+    const uint64_t s = seed ^ 0x5350454552ull;
+    uint32_t h = mix32((uint32_t)(s & 0xFFFFFFFFull) ^ kSeedPad);
+    h = mix32(h ^ (uint32_t)(s >> 32));
+    h = mix32(h ^ (uint32_t)(t & 0xFFFFFFFFull));
+    h = mix32(h ^ (uint32_t)(t >> 32));
+    h = mix32(h ^ stage);
+    std::vector<int> perm(n);
+    for (int i = 0; i < n; ++i) perm[i] = i;
+    for (int j = n - 1; j >= 1; --j) {
+        const uint32_t r = mix32(h ^ (uint32_t)j) % (uint32_t)(j + 1);
+        std::swap(perm[j], perm[r]);
+    }
+    std::vector<uint8_t> P((size_t)n * n);
+    for (int a = 0; a < n; ++a)
+        for (int b = 0; b < n; ++b) P[(size_t)a * n + b] = E[(size_t)perm[a] * n + perm[b]];
+    BlossomMatcher m(n, P);
+    const std::vector<int>& pm = m.solve();
+    mate.assign(n, -1);
+    int pairs = 0;
+    for (int a = 0; a < n; ++a) {
+        if (pm[a] != -1) {
+            mate[perm[a]] = perm[pm[a]];
+            pairs += pm[a] > a;
+        }
+    }
+    return pairs;
+}
+
+// FindConnectedSubgraph: component label per vertex; returns the number of components.
+int label_components(int n, const std::vector<uint8_t>& Q, std::vector<int>& label)
+{
+    label.assign(n, -1);
+    int c = 0;
+    std::vector<int> stack;
+    for (int s = 0; s < n; ++s) {
+        if (label[s] != -1) continue;
+        label[s] = c;
+        stack.push_back(s);
+        while (!stack.empty()) {
+            const int v = stack.back();
+            stack.pop_back();
+            for (int w = 0; w < n; ++w)
+                if (Q[(size_t)v * n + w] && label[w] == -1) {
+                    label[w] = c;
+                    stack.push_back(w);
+                }
+        }
+        ++c;
+    }
+    return c;
+}
+
+}  // namespace
+
+int select_peers(SelectState& st, const double* bandwidth, uint64_t t, int32_t* out_pairs)
+{
+    const int n = st.n;
+    if (t < st.last_t) return SAPS_ERR_INVALID;
+    for (int i = 0; i < n * n; ++i)
+        if (bandwidth[i] != bandwidth[i] || bandwidth[i] < 0.0) return SAPS_ERR_INVALID;
+
+    // B_ij = B_ji = min(B_ij, B_ji)
+    std::vector<double> B((size_t)n * n, 0.0);
+    for (int i = 0; i < n; ++i)
+        for (int j = 0; j < n; ++j)
+            if (i != j) B[(size_t)i * n + j] = std::min(bandwidth[(size_t)i * n + j], bandwidth[(size_t)j * n + i]);
+
+    double b_thres = st.b_thres;
+    if (st.b_thres_default) {
+        std::vector<double> links;
+        for (int i = 0; i < n; ++i)
+            for (int j = i + 1; j < n; ++j) links.push_back(B[(size_t)i * n + j]);
+        std::sort(links.begin(), links.end());
+        const size_t m = links.size();
+        b_thres = m == 0 ? 0.0 : (m % 2 ? links[m / 2] : 0.5 * (links[m / 2 - 1] + links[m / 2]));
+    }
+    int t_thres = st.t_thres;
+    if (t_thres == 0) {
+        int lg = 0;
+        while ((1 << lg) < n) ++lg;
+        t_thres = std::max(2, 2 * lg);
+    }
+
+    // IfConnected: recently connected edges, R_ij > t - T_thres
+    std::vector<uint8_t> Q((size_t)n * n, 0);
+    const int64_t horizon = (int64_t)t - (int64_t)t_thres;
+    for (int i = 0; i < n; ++i)
+        for (int j = 0; j < n; ++j) {
+            const int64_t r = st.R[(size_t)i * n + j];
+            if (i != j && r != kNever && r > horizon) Q[(size_t)i * n + j] = Q[(size_t)j * n + i] = 1;
+        }
+    std::vector<int> label;
+    const int ncomp = label_components(n, Q, label);
+
+    std::vector<uint8_t> E((size_t)n * n, 0);
+    for (int i = 0; i < n; ++i)
+        for (int j = 0; j < n; ++j) {
+            if (i == j) continue;
+            const double b = B[(size_t)i * n + j];
+            E[(size_t)i * n + j] = ncomp == 1 ? (b >= b_thres && b > 0.0)        // E = B*
+                                              : (label[i] != label[j] && b > 0.0);  // GetOverTimeMatrix
+        }
+
+    std::vector<int> mate;
+    const int first = randomly_max_match(n, E, st.seed, t, 1, mate);
+    if (2 * first != n) {
+        // GetUnmatch: every link between two still unmatched workers, bandwidth ignored
+        std::vector<uint8_t> E2((size_t)n * n, 0);
+        for (int i = 0; i < n; ++i)
+            for (int j = 0; j < n; ++j)
+                if (i != j && mate[i] == -1 && mate[j] == -1 && B[(size_t)i * n + j] > 0.0)
+                    E2[(size_t)i * n + j] = 1;
+        std::vector<int> mate2;
+        randomly_max_match(n, E2, st.seed, t, 2, mate2);
+        for (int i = 0; i < n; ++i)
+            if (mate2[i] != -1) mate[i] = mate2[i];
+    }
+
+    for (int i = 0; i < n; ++i) {
+        out_pairs[i] = mate[i] == -1 ? i : mate[i];
+        if (mate[i] != -1) st.R[(size_t)i * n + mate[i]] = (int64_t)t;
+    }
+    st.last_t = t;
+    return SAPS_OK;
+}
+
+}  // namespace saps

@@ -1,0 +1,267 @@
+"""CPU-side checks of the C-ABI library: it loads, exports what include/saps.h declares,
+validates arguments without touching a GPU, and its host-side peer selection agrees with
+the oracle and with brute force."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import peer_selection as ps
+from paper_2002_09692_b200 import binding as sb
+from paper_2002_09692_b200 import synth
+from helpers import all_perfect_matchings, check_involution, golden_records, max_matching_size_dp, parse_int
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "saps.h")).read()
+    return sorted(set(re.findall(r"SAPS_API[^;(]*?\b(saps_\w+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _declared()
+    assert len(names) >= 20 and "saps_round" in names and "saps_select_peers" in names
+    lib = ctypes.CDLL(str(sb._LIB_PATH))
+    for name in names:
+        assert hasattr(lib, name), f"{name} declared in saps.h but not exported"
+    assert sorted(sb.EXPORTS) == names, "binding and header disagree"
+
+
+def test_round_key_and_threshold_golden():
+    for rec in golden_records("mask_hash.txt"):
+        if rec[0] == "key":
+            assert sb.saps_round_key(parse_int(rec[1]), parse_int(rec[2])) == (parse_int(rec[3]), parse_int(rec[4]))
+        elif rec[0] == "thr":
+            assert sb.saps_threshold(float(rec[1])) == int(rec[2])
+    assert sb.saps_threshold(float("nan")) == 0 and sb.saps_threshold(7.0) == 1 << 32
+    # the library's host key and the oracle's agree on arbitrary inputs too
+    rng = np.random.default_rng(0)
+    for _ in range(200):
+        seed, t = int(rng.integers(0, 2 ** 63)), int(rng.integers(1, 2 ** 40))
+        assert sb.saps_round_key(seed, t) == oracle.round_key(seed, t)
+
+
+def test_create_validates():
+    for n, N, ld in ((0, 10, 10), (65, 10, 10), (4, 0, 0), (4, 1 << 32, 1 << 32), (4, 10, 9)):
+        with pytest.raises(sb.SapsError) as e:
+            sb.saps_create_ld(n, N, ld, 0)
+        assert e.value.status == sb.SAPS_ERR_INVALID
+    ctx = sb.saps_create_ld(64, (1 << 32) - 1, 1 << 32, 5)
+    sb.saps_destroy(ctx)
+    assert sb._lib.saps_destroy(None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_create(4, 10, 0, None) == sb.SAPS_ERR_INVALID
+
+
+def test_round_rejects_bad_arguments_before_any_launch():
+    # all of these fail on the host; no CUDA call is reached, so this runs without a GPU
+    ctx = sb.saps_create(4, 100, 0)
+    fake = 0x1000  # never dereferenced
+    good = [1, 0, 3, 2]
+
+    def status(**kw):
+        a = dict(x=fake, g=fake, lr=0.1, pairs=good, t=1, p=0.5)
+        a.update(kw)
+        return sb._lib.saps_round(ctx, a["x"], a["g"], a["lr"], sb._pairs(a["pairs"]), a["t"], a["p"], None)
+
+    assert status(x=None) == sb.SAPS_ERR_INVALID
+    assert status(t=0) == sb.SAPS_ERR_INVALID
+    assert status(p=-0.1) == sb.SAPS_ERR_INVALID
+    assert status(p=1.5) == sb.SAPS_ERR_INVALID
+    assert status(p=float("nan")) == sb.SAPS_ERR_INVALID
+    assert status(g=None, lr=0.1) == sb.SAPS_ERR_INVALID
+    assert status(lr=float("nan")) == sb.SAPS_ERR_INVALID
+    assert status(pairs=[1, 2, 0, 3]) == sb.SAPS_ERR_PAIRS
+    assert status(pairs=[1, 0, 4, 2]) == sb.SAPS_ERR_PAIRS
+    assert status(pairs=[-1, 0, 3, 2]) == sb.SAPS_ERR_PAIRS
+    assert sb._lib.saps_round(ctx, fake, fake, 0.1, None, 1, 0.5, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_pack(ctx, None, 1, 0.5, fake, fake, fake, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_pack(ctx, fake, 1, 0.5, None, fake, fake, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_pack(ctx, fake, 1, 2.0, fake, fake, fake, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_mask(ctx, 0, 0.5, fake, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_run_rounds(ctx, fake, fake, 0.1, 1, 3, 0.5, None, None, None, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_set_column_offset(ctx, (1 << 32) - 50) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_set_column_offset(ctx, (1 << 32) - 100) == sb.SAPS_OK
+    sb.saps_destroy(ctx)
+    for code in range(-6, 1):
+        assert sb.saps_strerror(code) not in ("", "unknown status")
+    assert sb.saps_strerror(-99) == "unknown status"
+
+
+def test_pack_capacity_formula():
+    ctx = sb.saps_create(32, 14_728_266, 0)
+    for p in (0.1, 0.01, 0.001):
+        phat = oracle.threshold(p) / 2.0 ** 32
+        N = 14_728_266
+        want = int(np.ceil(N * phat + 8 * np.sqrt(N * phat * (1 - phat)))) + 64
+        want = (want + 31) // 32 * 32
+        assert sb.saps_pack_capacity(ctx, p) == want
+        count = int(oracle.mask(0, 1, p, N).sum(dtype=np.int64))
+        assert count <= want
+    assert sb.saps_pack_capacity(ctx, 1.0) == 14_728_266
+    assert sb.saps_pack_capacity(ctx, 0.0) == 64
+    assert sb.saps_pack_capacity(ctx, float("nan")) == 0
+    sb.saps_set_pack_capacity(ctx, 1000)
+    assert sb.saps_pack_capacity(ctx, 0.5) == 1000
+    sb.saps_set_pack_capacity(ctx, 0)
+    assert sb.saps_pack_capacity(ctx, 1.0) == 14_728_266
+    sb.saps_destroy(ctx)
+
+
+# ---- host-side peer selection (Algorithm 3) against the oracle and brute force -------------
+
+def _candidate_edges(B, R, t, b_thres, t_thres):
+    E, mode = ps.candidate_edges(B, R, t, b_thres, t_thres)
+    return E, mode
+
+
+@pytest.mark.parametrize("n", [4, 6, 8])
+def test_select_peers_agrees_with_brute_force(n):
+    matchings = list(all_perfect_matchings(n))
+    for trial in range(20):
+        B = synth.bandwidth_matrix(n, 1.0, 100.0, seed=50 * n + trial)
+        ctx = sb.saps_create(n, 16, trial)
+        b_thres = ps.default_b_thres(B)
+        t_thres = ps.default_t_thres(n)
+        if trial % 2:
+            b_thres = 40.0 + trial
+            sb.saps_set_select_params(ctx, b_thres, 3)
+            t_thres = 3
+        R = ps.new_timestamps(n)                  # the oracle's copy of the state
+        for t in range(1, 14):
+            E, mode = _candidate_edges(B, R, t, b_thres, t_thres)
+            pairs = sb.saps_select_peers(ctx, B, t, n)
+            check_involution(pairs)
+            assert all(pairs[i] != i for i in range(n))
+            chosen = sum(1 for i in range(n) if pairs[i] > i and E[i, pairs[i]])
+            best = max(sum(1 for (a, b) in m if E[a, b]) for m in matchings)
+            assert chosen == best, (trial, t, mode)
+            # the oracle finds a matching of the same quality from the same state
+            _, info = ps.generate_gossip_matrix(B, R, t, b_thres, t_thres)
+            assert len(info["match"]) == chosen
+            ps.record_round(R, pairs, t)          # both sides continue from the library's choice
+            libR, last = sb.saps_get_select_state(ctx, n)
+            assert last == t
+            want = [[ps.NEVER if v == ps.NEVER else int(v) for v in row] for row in R]
+            assert [[sb.SAPS_NEVER if v == sb.SAPS_NEVER else v for v in row] for row in libR] == want
+        sb.saps_destroy(ctx)
+
+
+@pytest.mark.parametrize("n", [4, 6, 8])
+def test_select_peers_finds_planted_unique_optimum(n):
+    rng = np.random.default_rng(n)
+    for trial in range(8):
+        perm = rng.permutation(n)
+        planted = {(min(perm[a], perm[a + 1]), max(perm[a], perm[a + 1])) for a in range(0, n, 2)}
+        B = synth.bandwidth_matrix(n, 1.0, 10.0, seed=trial)
+        for i, j in planted:
+            B[i, j] = B[j, i] = 60.0
+        ctx = sb.saps_create(n, 16, trial)
+        sb.saps_set_select_params(ctx, 20.0, 5)
+        sb.saps_set_select_state(ctx, [[10 ** 6] * n for _ in range(n)], 10 ** 6)   # all recent
+        pairs = sb.saps_select_peers(ctx, B, 10 ** 6, n)
+        assert {(i, pairs[i]) for i in range(n) if pairs[i] > i} == planted
+        sb.saps_destroy(ctx)
+
+
+@pytest.mark.parametrize("n", [10, 14, 16, 32, 64])
+def test_select_peers_matching_size_against_independent_matchers(n):
+    # bandwidth mode on a sparse B*: compare the number of B* pairs with the subset DP (small n)
+    # and with the oracle's blossom (all n)
+    rng = np.random.default_rng(n)
+    for trial in range(6):
+        B = synth.bandwidth_matrix(n, 1.0, 100.0, seed=900 + trial)
+        b_thres = float(rng.choice([80.0, 90.0, 95.0]))
+        ctx = sb.saps_create(n, 16, trial)
+        sb.saps_set_select_params(ctx, b_thres, 4)
+        sb.saps_set_select_state(ctx, [[500] * n for _ in range(n)], 500)
+        R = np.full((n, n), 500, dtype=np.int64)
+        E, mode = _candidate_edges(B, R, 500, b_thres, 4)
+        assert mode == "bandwidth"
+        pairs = sb.saps_select_peers(ctx, B, 500, n)
+        check_involution(pairs)
+        assert all(pairs[i] != i for i in range(n))
+        chosen = sum(1 for i in range(n) if pairs[i] > i and E[i, pairs[i]])
+        assert chosen == len(ps.maximum_matching(E, rng.permutation(n)))
+        if n <= 16:
+            assert chosen == max_matching_size_dp(E.tolist())
+        sb.saps_destroy(ctx)
+
+
+def test_select_peers_schedule_invariants():
+    n = 32
+    B = synth.bandwidth_matrix(n, 1.0, 100.0, seed=1)
+    ctx = sb.saps_create(n, 16, 1)
+    b_thres, t_thres = ps.default_b_thres(B), ps.default_t_thres(n)
+    R = ps.new_timestamps(n)
+    S = ps.symmetrise(B)
+    connected_at, seen = [], set()
+    for t in range(1, 101):
+        label = ps.components(ps.recent_graph(R, t, t_thres))
+        pairs = sb.saps_select_peers(ctx, B, t, n)
+        check_involution(pairs)
+        assert all(pairs[i] != i for i in range(n))
+        seen.add(tuple(pairs))
+        if max(label) == 0:
+            connected_at.append(t)
+        else:
+            # merge mode: at least one pair joins two components, and as many as possible do
+            E, _ = ps.candidate_edges(B, R, t, b_thres, t_thres)
+            cross = sum(1 for i in range(n) if pairs[i] > i and label[i] != label[pairs[i]])
+            assert cross == len(ps.maximum_matching(E)) >= 1
+        ps.record_round(R, pairs, t)
+    later = [t for t in connected_at if t > 2 * t_thres]
+    assert later and np.diff([2 * t_thres] + later + [100]).max() <= t_thres
+    assert len(seen) > 50                      # the matching changes from round to round
+    # bandwidth mode prefers fast links: mean chosen bandwidth beats a random matching's mean
+    sb.saps_destroy(ctx)
+
+
+def test_select_peers_is_a_pure_function_of_seed_t_and_state():
+    n = 16
+    B = synth.bandwidth_matrix(n, 1.0, 100.0, seed=3)
+    a, b = sb.saps_create(n, 8, 7), sb.saps_create(n, 999, 7)
+    log_a = [sb.saps_select_peers(a, B, t, n) for t in range(1, 30)]
+    log_b = [sb.saps_select_peers(b, B, t, n) for t in range(1, 30)]
+    assert log_a == log_b
+    # checkpoint / resume reproduces the continuation
+    R, last = sb.saps_get_select_state(a, n)
+    cont = [sb.saps_select_peers(a, B, t, n) for t in range(30, 40)]
+    c = sb.saps_create(n, 8, 7)
+    sb.saps_set_select_state(c, R, last)
+    assert [sb.saps_select_peers(c, B, t, n) for t in range(30, 40)] == cont
+    # reset forgets
+    sb.saps_select_reset(a)
+    assert sb.saps_select_peers(a, B, 1, n) == log_a[0]
+    with pytest.raises(sb.SapsError):
+        sb.saps_select_peers(c, B, 5, n)       # t went backwards
+    for h in (a, b, c):
+        sb.saps_destroy(h)
+
+
+def test_select_peers_odd_n_missing_links_and_bad_input():
+    ctx = sb.saps_create(5, 8, 0)
+    B = synth.bandwidth_matrix(5, 1.0, 100.0, seed=4)
+    pairs = sb.saps_select_peers(ctx, B, 1, 5)
+    check_involution(pairs)
+    assert sum(1 for i in range(5) if pairs[i] == i) == 1
+    B[0, 1] = float("nan")
+    with pytest.raises(sb.SapsError):
+        sb.saps_select_peers(ctx, B, 2, 5)
+    sb.saps_destroy(ctx)
+    ctx = sb.saps_create(4, 8, 0)
+    B = synth.bandwidth_matrix(4, 1.0, 100.0, seed=4)
+    B[3, :] = B[:, 3] = 0.0
+    pairs = sb.saps_select_peers(ctx, B, 1, 4)
+    assert pairs[3] == 3 and sum(1 for i in range(4) if pairs[i] == i) == 2
+    # asymmetric input is symmetrised by the minimum
+    B2 = synth.bandwidth_matrix(4, 50.0, 100.0, seed=5)
+    B2[0, 1] = 1.0          # one direction slow: the link counts as slow
+    sb.saps_set_select_params(ctx, 40.0, 5)
+    sb.saps_set_select_state(ctx, [[9] * 4 for _ in range(4)], 9)
+    pairs = sb.saps_select_peers(ctx, B2, 9, 4)
+    assert pairs[0] != 1
+    sb.saps_destroy(ctx)

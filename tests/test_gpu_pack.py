@@ -1,0 +1,207 @@
+"""GPU parity of mask bitmap, compaction and the fused emission against the CPU oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2002_09692_b200 import synth
+from gpu_util import DeviceMatrix, assert_bits_equal, bits_from_mask, round_up, torch_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sb():
+    torch_cuda()
+    from paper_2002_09692_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("N", [1, 31, 32, 33, 255, 256, 257, 2048, 2049, 65_536, 272_474, 1_000_003])
+def test_mask_bitmap(sb, N):
+    torch = torch_cuda()
+    for seed, t, p in ((0, 1, 0.1), (1, 1, 0.01), (2, 20, 0.5), (0xDEADBEEFCAFEF00D, 2 ** 32 + 5, 0.001),
+                       (3, 3, 1.0), (3, 3, 0.0)):
+        words = round_up(N, 32) // 32
+        bits = torch.full((words + 2,), -1, dtype=torch.int32, device="cuda")
+        ctx = sb.saps_create(2, N, seed)
+        sb.saps_mask(ctx, t, p, bits)
+        torch.cuda.synchronize()
+        sb.saps_destroy(ctx)
+        got = bits.cpu().numpy().view(np.uint32)
+        want = bits_from_mask(oracle.mask(seed, t, p, N))
+        assert (got[:words] == want).all(), (N, seed, t, p)
+        assert (got[words:] == 0xFFFFFFFF).all()       # nothing written past the last word
+
+
+def test_mask_golden_columns_on_gpu(sb):
+    # the golden first/last kept columns of the tiny configuration come out of the CUDA hash
+    torch = torch_cuda()
+    N = 65_536
+    ctx = sb.saps_create(4, N, 0)
+    bits = torch.zeros(N // 32, dtype=torch.int32, device="cuda")
+    for t, count, first, last in ((1, 6617, [12, 15, 32, 40, 45, 70, 72, 111], 65520),
+                                  (2, 6765, [59, 68, 80, 116], 65528), (3, 6648, [0, 21, 43, 46], 65529)):
+        sb.saps_mask(ctx, t, 0.1, bits)
+        m = np.unpackbits(bits.cpu().numpy().view(np.uint8), bitorder="little")
+        idx = np.nonzero(m)[0]
+        assert len(idx) == count and list(idx[:len(first)]) == first and idx[-1] == last
+    sb.saps_destroy(ctx)
+
+
+def _pack_both(sb, n, N, ld, p, seed, t, with_idx=True, cap_override=0):
+    torch = torch_cuda()
+    x = synth.gaussian_matrix(n, N, 1.0, seed + 3, 0)
+    dx = DeviceMatrix(x, ld)
+    ctx = sb.saps_create_ld(n, N, ld, seed)
+    if cap_override:
+        sb.saps_set_pack_capacity(ctx, cap_override)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.full((n * cap + 32,), 123.0, dtype=torch.float32, device="cuda")
+    idx = torch.full((cap + 32,), -1, dtype=torch.int32, device="cuda")
+    count = torch.full((2,), -1, dtype=torch.int32, device="cuda")
+    sb.saps_pack(ctx, dx.ptr, t, p, vals, idx if with_idx else None, count)
+    torch.cuda.synchronize()
+    status = sb.saps_status(ctx)
+    sb.saps_destroy(ctx)
+    m = oracle.mask(seed, t, p, N)
+    wv, wi, wc = oracle.pack(x, m, cap)
+    got_count = int(count.cpu().numpy().view(np.uint32)[0])
+    assert got_count == wc, (N, p)
+    assert int(count[1]) == -1
+    k = min(wc, cap)
+    gv = vals.cpu().numpy()
+    gi = idx.cpu().numpy().view(np.uint32)
+    if with_idx:
+        assert (gi[:k] == wi[:k]).all()
+        assert (gi[k:] == 0xFFFFFFFF).all()              # slots past count untouched
+    else:
+        assert (gi == 0xFFFFFFFF).all()
+    got_vals = gv[:n * cap].reshape(n, cap)
+    assert_bits_equal(got_vals[:, :k], wv[:, :k], f"packed values N={N} p={p}")
+    assert (got_vals[:, k:] == 123.0).all() and (gv[n * cap:] == 123.0).all()
+    assert dx.canaries_intact()
+    return status, wc, cap
+
+
+@pytest.mark.parametrize("N", [1, 5, 33, 2047, 2048, 2049, 3 * 2048 + 1, 70_001])
+@pytest.mark.parametrize("p", [0.0, 0.01, 0.1, 0.5, 1.0])
+def test_pack_small(sb, N, p):
+    for n, ld in ((1, N), (4, N), (5, round_up(N, 32))):
+        status, _, _ = _pack_both(sb, n, N, ld, p, seed=N % 7, t=2)
+        assert status == 0
+
+
+def test_pack_many_tiles_and_no_index_list(sb):
+    # hundreds of tiles: the look-back crosses several 32-tile windows
+    for p in (0.001, 0.01, 0.1):
+        status, count, cap = _pack_both(sb, 8, 1_500_007, round_up(1_500_007, 32), p, seed=4, t=7)
+        assert status == 0 and count <= cap
+    status, _, _ = _pack_both(sb, 3, 300_000, 300_000, 0.05, seed=4, t=8, with_idx=False)
+    assert status == 0
+
+
+def test_pack_resnet20_shape(sb):
+    w = synth.WORKLOADS["resnet20"]
+    status, count, _ = _pack_both(sb, w.n, w.N, round_up(w.N, 32), 0.01, seed=1, t=1)
+    assert status == 0 and count == 2655                # golden count for seed 1, t 1
+
+
+def test_pack_overflow_is_reported_not_written(sb):
+    status, count, cap = _pack_both(sb, 4, 100_000, 100_000, 0.1, seed=2, t=1, cap_override=5000)
+    assert cap == 5000 and count > cap
+    assert status == sb.SAPS_ERR_OVERFLOW
+    # the status word is cleared by reading it: a clean call afterwards reports ok
+    status, _, _ = _pack_both(sb, 4, 100_000, 100_000, 0.1, seed=2, t=1)
+    assert status == 0
+
+
+def test_repeated_packs_reuse_the_scratch(sb):
+    torch = torch_cuda()
+    n, N, p = 4, 500_000, 0.02
+    x = synth.gaussian_matrix(n, N, 1.0, 8, 0)
+    dx = DeviceMatrix(x, N)
+    ctx = sb.saps_create(n, N, 8)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.zeros(n * cap, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    count = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for t in range(1, 8):
+        sb.saps_pack(ctx, dx.ptr, t, p, vals, idx, count)      # back to back, no sync
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    sb.saps_destroy(ctx)
+    m = oracle.mask(8, 7, p, N)
+    wv, wi, wc = oracle.pack(x, m, cap)
+    assert int(count[0]) == wc
+    assert (idx.cpu().numpy().view(np.uint32)[:wc] == wi[:wc]).all()
+    assert_bits_equal(vals.cpu().numpy().reshape(n, cap)[:, :wc], wv[:, :wc], "7th pack")
+
+
+@pytest.mark.parametrize("N,ld", [(7, 7), (2050, 2050), (2050, 2052), (40_003, 40_032), (40_003, 40_003),
+                                  (6 * 2048, 6 * 2048)])
+@pytest.mark.parametrize("p", [0.0, 0.05, 0.5, 1.0])
+@pytest.mark.parametrize("has_g", [True, False])
+def test_round_pack_emits_what_each_worker_sends(sb, N, ld, p, has_g):
+    torch = torch_cuda()
+    n = 6
+    pairs = [1, 0, 2, 5, 4, 3]                 # workers 2 and 4 have no peer
+    x = synth.gaussian_matrix(n, N, 1.0, 17, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, 17, 1) if has_g else None
+    lr = 0.1 if has_g else 0.0
+    dx = DeviceMatrix(x, ld)
+    dg = DeviceMatrix(g, ld) if has_g else None
+    ctx = sb.saps_create_ld(n, N, ld, 17)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.full((n * cap,), 123.0, dtype=torch.float32, device="cuda")
+    idx = torch.full((cap,), -1, dtype=torch.int32, device="cuda")
+    count = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    sb.saps_round_pack(ctx, dx.ptr, dg.ptr if has_g else None, lr, pairs, 5, p, vals, idx, count)
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    sb.saps_destroy(ctx)
+    a = x.copy()
+    oracle.sgd(a, g, lr)
+    m = oracle.mask(17, 5, p, N)
+    wv, wi, wc = oracle.pack(a, m, cap)
+    want = x.copy()
+    oracle.gossip_round(want, g, lr, pairs, 17, 5, p)
+    assert int(count.cpu().numpy().view(np.uint32)[0]) == wc
+    assert (idx.cpu().numpy().view(np.uint32)[:wc] == wi[:wc]).all()
+    got_vals = vals.cpu().numpy().reshape(n, cap)
+    assert_bits_equal(got_vals[:, :wc], wv[:, :wc], "emitted wire buffer")
+    assert (got_vals[:, wc:] == 123.0).all()
+    assert_bits_equal(dx.host(), want, "round result with emission")
+    assert dx.canaries_intact()
+
+
+def test_unfused_wire_path_equals_fused_round(sb):
+    # SGD-only round -> pack -> average the two packed buffers -> scatter  ==  fused round
+    torch = torch_cuda()
+    n, N, p, lr = 4, 50_000, 0.1, 0.05
+    pairs = [3, 2, 1, 0]
+    x = synth.gaussian_matrix(n, N, 1.0, 61, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, 61, 1)
+    ctx = sb.saps_create(n, N, 61)
+    fused, dg = DeviceMatrix(x, N), DeviceMatrix(g, N)
+    sb.saps_round(ctx, fused.ptr, dg.ptr, lr, pairs, 2, p)
+    unf = DeviceMatrix(x, N)
+    sb.saps_round(ctx, unf.ptr, dg.ptr, lr, list(range(n)), 2, p)        # SGD step only
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    count = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sb.saps_pack(ctx, unf.ptr, 2, p, vals, idx, count)
+    torch.cuda.synchronize()
+    c = int(count[0])
+    cols = idx[:c].long()
+    peer = torch.tensor(pairs, device="cuda")
+    merged = 0.5 * (vals[:, :c] + vals[peer, :c])
+    unf.view[:, :N].index_copy_(1, cols, merged)
+    assert_bits_equal(unf.host(), fused.host(), "wire path")
+    # after the round a worker and its peer hold identical kept coordinates
+    sb.saps_pack(ctx, fused.ptr, 2, p, vals, idx, count)
+    torch.cuda.synchronize()
+    v = vals.cpu().numpy()[:, :c]
+    for i in range(n):
+        assert_bits_equal(v[i], v[pairs[i]], "peers send identical buffers")
+    sb.saps_destroy(ctx)
