@@ -62,6 +62,7 @@ extern "C" {
 #define SAPS_ERR_OVERFLOW (-4)  /* more kept columns than the pack capacity (device-found) */
 #define SAPS_ERR_TIMEOUT  (-5)  /* the compaction scan gave up waiting (device-found)      */
 #define SAPS_ERR_NOMEM    (-6)  /* host or device allocation failed                        */
+#define SAPS_ERR_TOO_LARGE (-7) /* N beyond the static scratch of saps_pack_noalloc        */
 
 typedef struct saps_ctx saps_ctx;
 
@@ -143,6 +144,36 @@ SAPS_API int saps_set_pack_capacity(saps_ctx* ctx, uint64_t cap);
  * word is set to SAPS_ERR_OVERFLOW.  Slots r >= count are not written. */
 SAPS_API int saps_pack(saps_ctx* ctx, const float* x, uint64_t t, double keep_frac, float* out_vals,
               uint32_t* out_idx, uint32_t* out_count, void* stream);
+
+/* saps_pack for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for integration only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a serving or training
+ * process whose framework has already claimed the whole GPU for its own memory pool, a
+ * latency-critical loop that cannot afford the device-wide synchronisation an allocation
+ * implies, or a plug-in that is only handed buffers and a stream.  saps_pack would allocate
+ * the context's scratch area on its first use; this variant never does.  It calls neither
+ * cudaMalloc nor cudaFree nor any allocating library routine, now or later.
+ *
+ * Instead the tile states of the compaction scan live in a fixed array inside the library
+ * image (786,448 bytes, present on every GPU that loads the library, until the process
+ * exits).  That array covers N <= SAPS_NOALLOC_MAX_N columns; a larger context is refused
+ * with SAPS_ERR_TOO_LARGE before anything is launched.
+ *
+ * Arguments and results are those of saps_pack (same capacity rule, same overflow
+ * behaviour), plus
+ *   out_status  device, one int, or NULL: receives SAPS_OK, SAPS_ERR_OVERFLOW or
+ *               SAPS_ERR_TIMEOUT for this call (saps_status does not cover this entry point).
+ *
+ * The first call on each device looks up the array's device address (once per device, with
+ * that device current); make that first call outside any stream capture.  All calls, from
+ * all contexts, share the one array: it is cleared at the start of every call, and two
+ * calls that overlap on the same GPU (different streams, no ordering) race and give
+ * undefined results.  Calls on one stream, or ordered by events, are safe. */
+#define SAPS_NOALLOC_MAX_N 134217728ull
+SAPS_API int saps_pack_noalloc(saps_ctx* ctx, const float* x, uint64_t t, double keep_frac,
+                               float* out_vals, uint32_t* out_idx, uint32_t* out_count,
+                               int* out_status, void* stream);
 
 /* ---- peer selection (Algorithm 3; GetNewConnectedGraph of Algorithm 1) -------------------- */
 

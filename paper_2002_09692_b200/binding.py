@@ -22,6 +22,8 @@ SAPS_ERR_CUDA = -3
 SAPS_ERR_OVERFLOW = -4
 SAPS_ERR_TIMEOUT = -5
 SAPS_ERR_NOMEM = -6
+SAPS_ERR_TOO_LARGE = -7
+SAPS_NOALLOC_MAX_N = 134_217_728
 SAPS_NEVER = -(1 << 62)
 
 
@@ -51,6 +53,7 @@ _SIGNATURES = {
     "saps_pack_capacity": (_u64, [_vp, _f64]),
     "saps_set_pack_capacity": (_i32, [_vp, _u64]),
     "saps_pack": (_i32, [_vp, _vp, _u64, _f64, _vp, _vp, _vp, _vp]),
+    "saps_pack_noalloc": (_i32, [_vp, _vp, _u64, _f64, _vp, _vp, _vp, _vp, _vp]),
     "saps_set_select_params": (_i32, [_vp, _f64, _i32]),
     "saps_select_peers": (_i32, [_vp, _vp, _u64, _vp]),
     "saps_select_reset": (_i32, [_vp]),
@@ -167,6 +170,13 @@ def saps_set_pack_capacity(ctx, cap: int) -> None:
 def saps_pack(ctx, x, t, keep_frac, out_vals, out_idx, out_count, stream=None) -> None:
     _check(_lib.saps_pack(ctx, _ptr(x), t, keep_frac, _ptr(out_vals), _ptr(out_idx), _ptr(out_count),
                           _stream(stream)), "saps_pack")
+
+
+def saps_pack_noalloc(ctx, x, t, keep_frac, out_vals, out_idx, out_count, out_status=None, stream=None) -> None:
+    """saps_pack on the library's built-in scratch array: for callers that may not allocate
+    device memory.  Calls share that array, so keep them on one stream (or order them)."""
+    _check(_lib.saps_pack_noalloc(ctx, _ptr(x), t, keep_frac, _ptr(out_vals), _ptr(out_idx), _ptr(out_count),
+                                  _ptr(out_status), _stream(stream)), "saps_pack_noalloc")
 
 
 def saps_set_select_params(ctx, b_thres: float, t_thres: int) -> None:

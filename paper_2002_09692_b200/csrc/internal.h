@@ -102,6 +102,10 @@ cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream);
 cudaError_t launch_mask(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t* out_bits,
                         cudaStream_t stream);
 
+// Compaction on the library's static scratch area (no allocation anywhere on the path).
+constexpr uint32_t kStaticMaxTiles = 65536;  // kTileCols columns each: N <= 134,217,728
+cudaError_t launch_pack_static(PackArgs a, uint32_t ntiles, int* out_status, cudaStream_t stream);
+
 // ---- host-side peer selection (select_peers.cpp) ------------------------------------------
 
 struct SelectState {

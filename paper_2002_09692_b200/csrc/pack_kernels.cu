@@ -6,10 +6,17 @@
 // decoupled look-back over tile states orders the tiles.  Tiles take their number from an
 // atomic ticket, so every predecessor of a waiting tile is already running or done; the
 // wait is bounded all the same and ends with an error status, never a hang.
+#include <mutex>
+
 #include "internal.h"
 
 namespace saps {
 namespace {
+
+// Scratch of the allocation-free compaction entry point: the same layout as a context's
+// scratch (status word, ticket, tile states, tile prefixes) for up to kStaticMaxTiles column
+// tiles.  Every GPU that loads the library holds these bytes until the process exits.
+__device__ __align__(256) unsigned char g_static_scratch[16 + (size_t)kStaticMaxTiles * 12];
 
 constexpr unsigned long long kFlagAggregate = 1ull << 32;
 constexpr unsigned long long kFlagInclusive = 2ull << 32;
@@ -172,6 +179,47 @@ cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream)
     else
         pack_kernel<false><<<ntiles, kThreads, 0, stream>>>(a);
     return cudaGetLastError();
+}
+
+// In host code `g_static_scratch` names a host-side shadow of the device array, not device
+// memory; the address a kernel may use has to be asked for, per device, with that device
+// current.  It is looked up once per device and remembered.
+cudaError_t static_scratch_address(void** out)
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex lock;
+    static void* address[kMaxDevices] = {};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> hold(lock);
+    if (address[dev] == nullptr) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        address[dev] = p;
+    }
+    *out = address[dev];
+    return cudaSuccess;
+}
+
+cudaError_t launch_pack_static(PackArgs a, uint32_t ntiles, int* out_status, cudaStream_t stream)
+{
+    if (ntiles == 0 || ntiles > kStaticMaxTiles) return cudaErrorInvalidValue;
+    void* base = nullptr;
+    cudaError_t e = static_scratch_address(&base);
+    if (e != cudaSuccess) return e;
+    a.scratch = scratch_view(base, ntiles);
+    // the area keeps whatever the previous call left: status, ticket and tile states restart at zero
+    e = cudaMemsetAsync(base, 0, 4 + scratch_clear_bytes(ntiles), stream);
+    if (e != cudaSuccess) return e;
+    pack_kernel<true><<<ntiles, kThreads, 0, stream>>>(a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (out_status != nullptr)
+        e = cudaMemcpyAsync(out_status, a.scratch.status, sizeof(int), cudaMemcpyDeviceToDevice, stream);
+    return e;
 }
 
 cudaError_t launch_mask(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t* out_bits,

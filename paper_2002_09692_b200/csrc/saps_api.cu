@@ -289,6 +289,32 @@ int saps_pack(saps_ctx* ctx, const float* x, uint64_t t, double keep_frac, float
     return launch_pack(a, (cudaStream_t)stream) == cudaSuccess ? SAPS_OK : SAPS_ERR_CUDA;
 }
 
+int saps_pack_noalloc(saps_ctx* ctx, const float* x, uint64_t t, double keep_frac, float* out_vals,
+                      uint32_t* out_idx, uint32_t* out_count, int* out_status, void* stream)
+{
+    if (ctx == nullptr || x == nullptr || out_vals == nullptr || out_count == nullptr || t == 0 ||
+        !valid_frac(keep_frac))
+        return SAPS_ERR_INVALID;
+    if (ctx->N > SAPS_NOALLOC_MAX_N) return SAPS_ERR_TOO_LARGE;
+    PackArgs a;
+    a.x = x;
+    a.ld = (size_t)ctx->ld;
+    a.N = (uint32_t)ctx->N;
+    a.n = ctx->n;
+    a.key = make_key(ctx->seed, t, keep_frac);
+    a.col_offset = (uint32_t)ctx->col_offset;
+    a.cap = (uint32_t)saps_pack_capacity(ctx, keep_frac);
+    a.out_vals = out_vals;
+    a.out_idx = out_idx;
+    a.out_count = out_count;
+    a.spin_limit = kSpinLimit;
+    if (launch_pack_static(a, ctx->ntiles, out_status, (cudaStream_t)stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SAPS_ERR_CUDA;
+    }
+    return SAPS_OK;
+}
+
 int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, const int32_t* pairs,
                     uint64_t t, double keep_frac, float* out_vals, uint32_t* out_idx,
                     uint32_t* out_count, void* stream)
@@ -478,6 +504,7 @@ const char* saps_strerror(int status)
         case SAPS_ERR_OVERFLOW: return "more kept columns than the pack capacity";
         case SAPS_ERR_TIMEOUT: return "compaction scan gave up waiting for a predecessor tile";
         case SAPS_ERR_NOMEM: return "out of memory";
+        case SAPS_ERR_TOO_LARGE: return "N exceeds what the static scratch area of saps_pack_noalloc covers";
         default: return "unknown status";
     }
 }
