@@ -30,6 +30,10 @@ if ROOT not in sys.path:
 METRIC = "gossip_rounds_per_s"
 UNIT = "rounds/s"
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes (read + write) per worker-parameter of the fused round kernel, from the ncu
+# capture summarised in profiles/round_kernel_mnistcnn_ncu.md (traffic grows in proportion
+# to n*N).  Set to None whenever round_kernels.cu changes until the counters are retaken.
+NCU_TRAFFIC_BYTES_PER_ELEMENT = 11.792
 
 
 def parse_args():
@@ -284,7 +288,8 @@ def run_ours(args):
             "bound": "hbm", "kernel": "round_kernel<4,true,true> (fused SGD + mask + emit + pair average)",
             "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
             "frac": achieved / peak, "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
-            "kernel_ms": k_ms, "algorithmic_bytes": bytes_round + bytes_emit, "traffic": None,
+            "kernel_ms": k_ms, "algorithmic_bytes": bytes_round + bytes_emit,
+            "traffic": None if NCU_TRAFFIC_BYTES_PER_ELEMENT is None else NCU_TRAFFIC_BYTES_PER_ELEMENT * n * N,
         },
     }
 

@@ -35,6 +35,9 @@ WORKLOADS = {
     "tiny": Workload("tiny", 4, 65_536, 1.0, 0.01, 0.1, (0.1,), 3, 0, "fixed",
                      fixed_pairs=(1, 0, 3, 2)),
     "resnet20": Workload("resnet20", 32, 272_474, 0.05, 0.01, 0.1, (0.01,), 100, 1, "select"),
+    # the paper's own model sizes (Table 2) with its c = 100
+    "mnistcnn": Workload("mnistcnn", 32, 6_653_628, 0.05, 0.01, 0.05, (0.01,), 50, 0, "select"),
+    "cifar10cnn": Workload("cifar10cnn", 32, 7_025_886, 0.05, 0.01, 0.04, (0.01,), 50, 0, "select"),
     "vgg16": Workload("vgg16", 32, 14_728_266, 0.05, 0.01, 0.05, (0.01, 0.001), 50, 0, "select"),
     "resnet50": Workload("resnet50", 32, 25_557_032, 0.05, 0.01, 0.05,
                          (0.1, 0.03, 0.01, 0.003, 0.001), 20, 2, "random"),
