@@ -31,7 +31,7 @@ METRIC = "gossip_rounds_per_s"
 UNIT = "rounds/s"
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per worker-parameter of the fused round kernel, from the ncu
-# capture summarised in profiles/round_kernel_mnistcnn_ncu.md (traffic grows in proportion
+# capture of that kernel on a smaller workload (summary under profiles/; traffic grows in proportion
 # to n*N).  Set to None whenever round_kernels.cu changes until the counters are retaken.
 NCU_TRAFFIC_BYTES_PER_ELEMENT = 11.792
 
