@@ -72,7 +72,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "100", "-i", str(gpu_index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                 "-lms", "20", "-i", str(gpu_index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             pass
 
@@ -178,7 +178,7 @@ def run_ours(args):
     import torch
 
     from paper_2002_09692_b200 import binding as sb
-    from paper_2002_09692_b200 import synth
+    from paper_2002_09692_b200 import sharding, synth
 
     rank, world, local = dist_env()
     if not torch.cuda.is_available():
@@ -205,7 +205,8 @@ def run_ours(args):
     B = synth.bandwidth_matrix(n, *w.bw_range, seed=w.seed)
 
     ctx = sb.saps_create_ld(n, N, ld, w.seed)
-    sb.saps_set_column_offset(ctx, rank * N)
+    col_offset, _ = sharding.weak_shard(N, world, rank)
+    sb.saps_set_column_offset(ctx, col_offset)
     cap = sb.saps_pack_capacity(ctx, p)
     vals = torch.empty(n, cap, dtype=torch.float32, device="cuda")
     idx = torch.empty(cap, dtype=torch.int32, device="cuda")
@@ -255,10 +256,7 @@ def run_ours(args):
     elapsed_ms = ev_start.elapsed_time(ev_stop)
     kernel_ms = [a.elapsed_time(b) for a, b in zip(ev_k0, ev_k1)]
     kept = int(count.cpu().numpy().view(np.uint32)[0])
-    if world > 1:
-        tm = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tm.item())
+    elapsed_ms = sharding.max_over_ranks(elapsed_ms)
 
     ms_per_step = elapsed_ms / K
     value = world * K / (elapsed_ms * 1e-3)
@@ -316,19 +314,33 @@ def measure_e2e(args, sb, synth, w, ctx, B, t, x_dev, g_dev):
     hx.copy_(x_dev[:, :N])
     hg.copy_(g_dev[:, :N])
     sb.saps_set_column_offset(ctx, 0)
+    cap = sb.saps_pack_capacity(ctx, args.keep_frac)
+    hv = torch.empty(n, cap, dtype=torch.float32).pin_memory()
+    hi = torch.empty(cap, dtype=torch.int32).pin_memory()
+    hc = torch.zeros(1, dtype=torch.int32).pin_memory()
+    d_v = torch.empty(n, cap, dtype=torch.float32, device="cuda")
+    d_i = torch.empty(cap, dtype=torch.int32, device="cuda")
+    d_c = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def step(t):
+        sb.saps_round_pack_host(ctx, hx, hg, w.lr, sb.saps_select_peers(ctx, B, t, n), t, args.keep_frac,
+                                x_dev, g_dev, hv, hi, hc, d_v, d_i, d_c)
+
     steps = max(1, args.e2e_steps)
     for _ in range(2):
-        sb.saps_round_host(ctx, hx, hg, w.lr, sb.saps_select_peers(ctx, B, t, n), t, args.keep_frac, x_dev, g_dev)
+        step(t)
         t += 1
     torch.cuda.synchronize()
     t0 = time.perf_counter()
     for _ in range(steps):
-        sb.saps_round_host(ctx, hx, hg, w.lr, sb.saps_select_peers(ctx, B, t, n), t, args.keep_frac, x_dev, g_dev)
+        step(t)
         t += 1
     dt = time.perf_counter() - t0                     # the call waits for the copies back
     return {"value": steps / dt, "unit": UNIT, "h2d_bytes_per_step": 2 * 4 * n * N,
-            "d2h_bytes_per_step": 4 * n * N, "ms_per_step": dt / steps * 1e3, "steps": steps,
-            "api": "saps_select_peers + saps_round_host (pinned host x and g in, x out; chunked copy/compute pipeline)"}
+            "d2h_bytes_per_step": 4 * n * N + 4 * n * cap + 4 * cap + 4, "ms_per_step": dt / steps * 1e3,
+            "steps": steps, "kept_columns": int(hc.numpy().view("uint32")[0]),
+            "api": "saps_select_peers + saps_round_pack_host (pinned host x and g in; x, packed values, "
+                   "indices and count out; chunked copy/compute pipeline over 3 streams)"}
 
 
 def measure_cpu_baseline(args, synth, w):

@@ -224,6 +224,16 @@ SAPS_API int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, 
 SAPS_API int saps_round_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
                     const int32_t* pairs, uint64_t t, double keep_frac, float* d_x, float* d_g);
 
+/* The same with the wire buffer of step 3 (as saps_round_pack): out_vals_host [n, cap],
+ * out_idx_host [cap] or NULL, out_count_host (one word) are HOST buffers filled before the
+ * call returns; d_vals [n, cap], d_idx [cap], d_count are device staging (d_idx may be NULL
+ * when out_idx_host is).  cap = saps_pack_capacity(ctx, keep_frac). */
+SAPS_API int saps_round_pack_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
+                                  const int32_t* pairs, uint64_t t, double keep_frac, float* d_x,
+                                  float* d_g, float* out_vals_host, uint32_t* out_idx_host,
+                                  uint32_t* out_count_host, float* d_vals, uint32_t* d_idx,
+                                  uint32_t* d_count);
+
 /* ---- measurement ------------------------------------------------------------------------------- */
 
 /* Optional cudaEvent_t pair (as void*; NULL, NULL switches it off).  When set, saps_round

@@ -61,6 +61,7 @@ _SIGNATURES = {
     "saps_set_select_state": (_i32, [_vp, _vp, _u64]),
     "saps_run_rounds": (_i32, [_vp, _vp, _vp, _f32, _u64, _u64, _f64, _vp, _vp, _vp, _vp]),
     "saps_round_host": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp, _vp]),
+    "saps_round_pack_host": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "saps_set_timing_events": (_i32, [_vp, _vp, _vp]),
     "saps_status": (_i32, [_vp, _vp, ctypes.POINTER(_i32)]),
     "saps_strerror": (ctypes.c_char_p, [_i32]),
@@ -230,6 +231,14 @@ def saps_run_rounds(ctx, x, g, lr, t_first, T, keep_frac, pairs_list=None, bandw
 def saps_round_host(ctx, x_host, g_host, lr, pairs, t, keep_frac, d_x, d_g) -> None:
     _check(_lib.saps_round_host(ctx, _ptr(x_host), _ptr(g_host), lr, _pairs(pairs), t, keep_frac,
                                 _ptr(d_x), _ptr(d_g)), "saps_round_host")
+
+
+def saps_round_pack_host(ctx, x_host, g_host, lr, pairs, t, keep_frac, d_x, d_g, out_vals_host,
+                         out_idx_host, out_count_host, d_vals, d_idx, d_count) -> None:
+    _check(_lib.saps_round_pack_host(ctx, _ptr(x_host), _ptr(g_host), lr, _pairs(pairs), t, keep_frac,
+                                     _ptr(d_x), _ptr(d_g), _ptr(out_vals_host), _ptr(out_idx_host),
+                                     _ptr(out_count_host), _ptr(d_vals), _ptr(d_idx), _ptr(d_count)),
+           "saps_round_pack_host")
 
 
 def saps_set_timing_events(ctx, before, after) -> None:

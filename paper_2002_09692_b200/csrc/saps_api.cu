@@ -25,6 +25,7 @@ struct saps_ctx {
     // pipeline of the host-buffer entry point, created on first use
     static constexpr int kLanes = 3;
     cudaStream_t lane_stream[kLanes];
+    cudaEvent_t lane_event[kLanes];
     bool lanes_ready;
     SelectState select;
 };
@@ -198,7 +199,10 @@ int saps_destroy(saps_ctx* ctx)
 {
     if (ctx == nullptr) return SAPS_ERR_INVALID;
     if (ctx->lanes_ready)
-        for (int l = 0; l < saps_ctx::kLanes; ++l) cudaStreamDestroy(ctx->lane_stream[l]);
+        for (int l = 0; l < saps_ctx::kLanes; ++l) {
+            cudaStreamDestroy(ctx->lane_stream[l]);
+            cudaEventDestroy(ctx->lane_event[l]);
+        }
     if (ctx->scratch != nullptr) cudaFree(ctx->scratch);
     delete ctx;
     return SAPS_OK;
@@ -420,34 +424,89 @@ int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t 
     return SAPS_OK;
 }
 
-int saps_round_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr, const int32_t* pairs,
-                    uint64_t t, double keep_frac, float* d_x, float* d_g)
+namespace {
+
+// Optional wire-buffer outputs of the host-buffer entry point.
+struct HostPack {
+    float* vals_host;      // [n, cap]
+    uint32_t* idx_host;    // [cap] or NULL
+    uint32_t* count_host;  // one word
+    float* d_vals;         // device staging
+    uint32_t* d_idx;
+    uint32_t* d_count;
+};
+
+int ensure_lanes(saps_ctx* ctx)
+{
+    if (ctx->lanes_ready) return SAPS_OK;
+    int ns = 0, ne = 0;
+    while (ns < saps_ctx::kLanes &&
+           cudaStreamCreateWithFlags(&ctx->lane_stream[ns], cudaStreamNonBlocking) == cudaSuccess)
+        ++ns;
+    while (ns == saps_ctx::kLanes && ne < saps_ctx::kLanes &&
+           cudaEventCreateWithFlags(&ctx->lane_event[ne], cudaEventDisableTiming) == cudaSuccess)
+        ++ne;
+    if (ne != saps_ctx::kLanes) {
+        for (int m = 0; m < ne; ++m) cudaEventDestroy(ctx->lane_event[m]);
+        for (int m = 0; m < ns; ++m) cudaStreamDestroy(ctx->lane_stream[m]);
+        cudaGetLastError();
+        return SAPS_ERR_CUDA;
+    }
+    ctx->lanes_ready = true;
+    return SAPS_OK;
+}
+
+// The round acts column by column, so column chunks are independent: copy in, compute and
+// copy out chunk by chunk, round-robin over a few streams, so that the two copy directions
+// and the kernels overlap.  With a wire buffer, the mask scan (which touches no model data)
+// runs first on lane 0 and the other lanes wait for its tile prefixes.
+int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr, const int32_t* pairs,
+                    uint64_t t, double keep_frac, float* d_x, float* d_g, const HostPack* pack)
 {
     int rc = check_round_args(ctx, x_host, g_host, lr, t, keep_frac);
     if (rc != SAPS_OK) return rc;
     if (d_x == nullptr || (g_host != nullptr && d_g == nullptr)) return SAPS_ERR_INVALID;
+    if (pack != nullptr && (pack->vals_host == nullptr || pack->count_host == nullptr || pack->d_vals == nullptr ||
+                            pack->d_count == nullptr || (pack->idx_host != nullptr && pack->d_idx == nullptr)))
+        return SAPS_ERR_INVALID;
     rc = check_pairs(ctx->n, pairs);
     if (rc != SAPS_OK) return rc;
-    if (!ctx->lanes_ready) {
-        for (int l = 0; l < saps_ctx::kLanes; ++l) {
-            if (cudaStreamCreateWithFlags(&ctx->lane_stream[l], cudaStreamNonBlocking) != cudaSuccess) {
-                for (int m = 0; m < l; ++m) cudaStreamDestroy(ctx->lane_stream[m]);
-                cudaGetLastError();
-                return SAPS_ERR_CUDA;
-            }
-        }
-        ctx->lanes_ready = true;
+    rc = ensure_lanes(ctx);
+    if (rc != SAPS_OK) return rc;
+    if (pack != nullptr) {
+        rc = ensure_scratch(ctx);
+        if (rc != SAPS_OK) return rc;
     }
     const int n = ctx->n;
     const uint64_t N = ctx->N;
     const uint64_t ld_dev = (N + 31) / 32 * 32;
-    // The round acts column by column, so column chunks are independent: copy in, compute
-    // and copy out chunk by chunk, round-robin over a few streams, so that the two copy
-    // directions and the kernel overlap.
-    const RowGroups rg = make_groups(n, pairs, g_host != nullptr);
+    const bool emit = pack != nullptr;
+    const RowGroups rg = make_groups(n, pairs, g_host != nullptr || emit);
     const RoundKey key = make_key(ctx->seed, t, keep_frac);
-    const uint32_t tiles_per_chunk = 512;  // 1 Mi columns: n x 4 MiB per matrix and chunk
+    const uint32_t cap = emit ? (uint32_t)saps_pack_capacity(ctx, keep_frac) : 0;
     bool failed = false;
+    ScratchView sv{};
+    if (emit) {
+        sv = scratch_view(ctx->scratch, ctx->ntiles);
+        PackArgs p;
+        p.x = nullptr;
+        p.ld = (size_t)ld_dev;
+        p.N = (uint32_t)N;
+        p.n = n;
+        p.key = key;
+        p.col_offset = (uint32_t)ctx->col_offset;
+        p.cap = cap;
+        p.out_vals = nullptr;
+        p.out_idx = pack->idx_host != nullptr ? pack->d_idx : nullptr;
+        p.out_count = pack->d_count;
+        p.scratch = sv;
+        p.spin_limit = kSpinLimit;
+        failed |= launch_pack(p, ctx->lane_stream[0]) != cudaSuccess;
+        failed |= cudaEventRecord(ctx->lane_event[0], ctx->lane_stream[0]) != cudaSuccess;
+        for (int l = 1; l < saps_ctx::kLanes; ++l)
+            failed |= cudaStreamWaitEvent(ctx->lane_stream[l], ctx->lane_event[0], 0) != cudaSuccess;
+    }
+    const uint32_t tiles_per_chunk = 512;  // 1 Mi columns: n x 4 MiB per matrix and chunk
     int lane = 0;
     for (uint32_t tb = 0; tb < ctx->ntiles && !failed; tb += tiles_per_chunk, lane = (lane + 1) % saps_ctx::kLanes) {
         const uint32_t tc = ctx->ntiles - tb < tiles_per_chunk ? ctx->ntiles - tb : tiles_per_chunk;
@@ -463,9 +522,29 @@ int saps_round_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
         RoundArgs a = round_args(ctx, d_x, g_host != nullptr ? d_g : nullptr, lr, rg, key, ld_dev);
         a.tile_begin = tb;
         a.tile_count = tc;
-        failed |= launch_round(a, false, s) != cudaSuccess;
+        if (emit) {
+            a.out_vals = pack->d_vals;
+            a.cap = cap;
+            a.tile_excl = sv.tile_excl;
+        }
+        failed |= launch_round(a, emit, s) != cudaSuccess;
         failed |= cudaMemcpy2DAsync(x_host + c0, N * sizeof(float), d_x + c0, ld_dev * sizeof(float), width, n,
                                     cudaMemcpyDeviceToHost, s) != cudaSuccess;
+    }
+    if (emit && !failed) {
+        // the wire buffer is complete once every lane has run its chunks
+        cudaStream_t s0 = ctx->lane_stream[0];
+        for (int l = 1; l < saps_ctx::kLanes; ++l) {
+            failed |= cudaEventRecord(ctx->lane_event[l], ctx->lane_stream[l]) != cudaSuccess;
+            failed |= cudaStreamWaitEvent(s0, ctx->lane_event[l], 0) != cudaSuccess;
+        }
+        failed |= cudaMemcpyAsync(pack->count_host, pack->d_count, sizeof(uint32_t), cudaMemcpyDeviceToHost, s0) !=
+                  cudaSuccess;
+        failed |= cudaMemcpyAsync(pack->vals_host, pack->d_vals, (size_t)n * cap * sizeof(float),
+                                  cudaMemcpyDeviceToHost, s0) != cudaSuccess;
+        if (pack->idx_host != nullptr)
+            failed |= cudaMemcpyAsync(pack->idx_host, pack->d_idx, (size_t)cap * sizeof(uint32_t),
+                                      cudaMemcpyDeviceToHost, s0) != cudaSuccess;
     }
     for (int l = 0; l < saps_ctx::kLanes; ++l) failed |= cudaStreamSynchronize(ctx->lane_stream[l]) != cudaSuccess;
     if (failed) {
@@ -473,6 +552,23 @@ int saps_round_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
         return SAPS_ERR_CUDA;
     }
     return SAPS_OK;
+}
+
+}  // namespace
+
+int saps_round_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr, const int32_t* pairs,
+                    uint64_t t, double keep_frac, float* d_x, float* d_g)
+{
+    return round_host_impl(ctx, x_host, g_host, lr, pairs, t, keep_frac, d_x, d_g, nullptr);
+}
+
+int saps_round_pack_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr, const int32_t* pairs,
+                         uint64_t t, double keep_frac, float* d_x, float* d_g, float* out_vals_host,
+                         uint32_t* out_idx_host, uint32_t* out_count_host, float* d_vals, uint32_t* d_idx,
+                         uint32_t* d_count)
+{
+    const HostPack pack{out_vals_host, out_idx_host, out_count_host, d_vals, d_idx, d_count};
+    return round_host_impl(ctx, x_host, g_host, lr, pairs, t, keep_frac, d_x, d_g, &pack);
 }
 
 int saps_status(saps_ctx* ctx, void* stream, int* out_device_status)

@@ -249,3 +249,37 @@ def test_round_host_entry_point(sb):
     oracle.gossip_round(want2, None, 0.0, pairs, 51, 3, p)
     assert_bits_equal(hx2.numpy(), want2, "host entry point, no gradient")
     sb.saps_destroy(ctx)
+
+
+def test_round_pack_host_entry_point(sb):
+    torch = torch_cuda()
+    n, N, p = 6, 2_300_000, 0.01
+    x = synth.gaussian_matrix(n, N, 0.05, 52, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, 52, 1)
+    pairs = [1, 0, 3, 2, 5, 4]
+    ctx = sb.saps_create(n, N, 52)
+    cap = sb.saps_pack_capacity(ctx, p)
+    ld = round_up(N, 32)
+    hx = torch.from_numpy(x.copy()).pin_memory()
+    hg = torch.from_numpy(g).pin_memory()
+    hv = torch.full((n, cap), 123.0, dtype=torch.float32).pin_memory()
+    hi = torch.full((cap,), -1, dtype=torch.int32).pin_memory()
+    hc = torch.full((1,), -1, dtype=torch.int32).pin_memory()
+    d_x = torch.empty(n * ld, dtype=torch.float32, device="cuda")
+    d_g = torch.empty(n * ld, dtype=torch.float32, device="cuda")
+    d_v = torch.empty(n * cap, dtype=torch.float32, device="cuda")
+    d_i = torch.empty(cap, dtype=torch.int32, device="cuda")
+    d_c = torch.empty(1, dtype=torch.int32, device="cuda")
+    sb.saps_round_pack_host(ctx, hx, hg, 0.05, pairs, 4, p, d_x, d_g, hv, hi, hc, d_v, d_i, d_c)
+    assert sb.saps_status(ctx) == 0
+    sb.saps_destroy(ctx)
+    a = x.copy()
+    oracle.sgd(a, g, 0.05)
+    m = oracle.mask(52, 4, p, N)
+    wv, wi, wc = oracle.pack(a, m, cap)
+    want = x.copy()
+    oracle.gossip_round(want, g, 0.05, pairs, 52, 4, p)
+    assert int(hc[0]) == wc
+    assert (hi.numpy().view(np.uint32)[:wc] == wi[:wc]).all()
+    assert_bits_equal(hv.numpy()[:, :wc], wv[:, :wc], "host wire buffer")
+    assert_bits_equal(hx.numpy(), want, "host entry point with wire buffer")

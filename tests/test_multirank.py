@@ -1,0 +1,82 @@
+"""The N > 1 path on CPU: two gloo ranks exercise the host logic that bench.py --gpus N uses
+(column shards, identical matchings on every rank without communication, global placement of
+the packed buffers, max-over-ranks timing)."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import oracle
+from paper_2002_09692_b200 import sharding, synth
+
+
+def test_column_shard_covers_everything_once():
+    for n_total in (1, 2047, 2048, 2049, 14_728_266, 124_439_808):
+        for world in (1, 2, 3, 8):
+            spans = [sharding.column_shard(n_total, world, r) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == n_total
+            for (b0, e0), (b1, e1) in zip(spans, spans[1:]):
+                assert e0 == b1 and b0 <= e0
+            for b, e in spans:
+                assert b % sharding.TILE_COLS == 0 or b == n_total
+            sizes = [e - b for b, e in spans]
+            assert max(sizes) - min(sizes) <= 2 * sharding.TILE_COLS
+    with pytest.raises(ValueError):
+        sharding.weak_shard(1 << 30, 8, 0)
+    assert sharding.weak_shard(14_728_266, 8, 7) == (7 * 14_728_266, 14_728_266)
+    assert sharding.exclusive_offsets([3, 0, 5]) == ([0, 3, 3], 8)
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, n_total, results):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        from paper_2002_09692_b200 import binding as sb
+        n, seed, p, T = 8, 3, 0.05, 6
+        begin, end = sharding.column_shard(n_total, world, rank)
+        # every rank selects its peers on its own: same seed, t and bandwidth -> same matching
+        B = synth.bandwidth_matrix(n, 1.0, 100.0, seed=seed)
+        ctx = sb.saps_create(n, max(1, end - begin), seed)
+        sb.saps_set_column_offset(ctx, begin)
+        mine = [sb.saps_select_peers(ctx, B, t, n) for t in range(1, T + 1)]
+        sb.saps_destroy(ctx)
+        gathered = [None] * world
+        dist.all_gather_object(gathered, mine)
+        assert all(g == gathered[0] for g in gathered), "ranks disagree on the matching"
+        # this shard's part of the round mask and its place in the global wire buffer
+        m = oracle.mask(seed, 1, p, n_total)[begin:end]
+        offset, total = sharding.global_pack_offset(int(m.sum()))
+        slowest = sharding.max_over_ranks(10.0 + rank)
+        results[rank] = (begin, end, int(m.sum()), offset, total, slowest)
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_gloo():
+    world, n_total = 2, 5 * 2048 + 300
+    ctx = mp.get_context("spawn")
+    with ctx.Manager() as mgr:
+        results = mgr.dict()
+        port = _free_port()
+        procs = [ctx.Process(target=_worker, args=(r, world, port, n_total, results)) for r in range(world)]
+        for pr in procs:
+            pr.start()
+        for pr in procs:
+            pr.join(120)
+            assert pr.exitcode == 0
+        res = [results[r] for r in range(world)]
+    full = oracle.mask(3, 1, 0.05, n_total)
+    assert res[0][0] == 0 and res[0][1] == res[1][0] and res[1][1] == n_total
+    assert res[0][3] == 0 and res[1][3] == res[0][2]                    # exclusive scan of the counts
+    assert res[0][4] == res[1][4] == int(full.sum()) == res[0][2] + res[1][2]
+    assert res[0][5] == res[1][5] == 11.0                               # the slowest rank's time
