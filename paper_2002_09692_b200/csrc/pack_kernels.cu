@@ -33,6 +33,58 @@ __device__ __forceinline__ uint32_t warp_sum(uint32_t v)
     return v;
 }
 
+// Decoupled look-back, run by one full warp: publishes this tile's count, sums the counts of
+// all earlier tiles (32 tile states per step), then publishes the inclusive prefix.
+// Returns false when a predecessor did not publish within the poll budget (or another tile
+// already reported an error); the status word then holds SAPS_ERR_TIMEOUT.
+__device__ __forceinline__ bool lookback_exclusive(const ScratchView& sc, uint32_t tile, uint32_t total,
+                                                   uint32_t spin_limit, int lane, uint32_t* out_excl)
+{
+    if (lane == 0)
+        atomicExch(&sc.tile_state[tile], (tile == 0 ? kFlagInclusive : kFlagAggregate) | total);
+    uint32_t excl = 0;
+    bool ok = true;
+    if (tile > 0) {
+        long long look = (long long)tile - 1;  // newest tile of the window
+        uint32_t polls = 0;
+        while (true) {
+            const long long idx = look - lane;
+            // tiles before the first count as "inclusive prefix 0"
+            const unsigned long long st = idx >= 0 ? peek_state(&sc.tile_state[idx]) : kFlagInclusive;
+            const uint32_t flag = (uint32_t)(st >> 32);
+            const uint32_t incl = __ballot_sync(0xFFFFFFFFu, flag == 2u);
+            const uint32_t empty = __ballot_sync(0xFFFFFFFFu, flag == 0u);
+            const int first = incl ? (__ffs(incl) - 1) : 32;  // nearest inclusive prefix
+            const uint32_t needed = first >= 31 ? 0xFFFFFFFFu : ((2u << first) - 1u);
+            if (empty & needed) {
+                // a predecessor has not published yet: back off and poll again
+                ++polls;
+                bool give_up = polls > spin_limit;
+                if ((polls & 63u) == 0u) give_up |= *reinterpret_cast<volatile int*>(sc.status) != 0;
+                if (__any_sync(0xFFFFFFFFu, give_up)) {
+                    ok = false;
+                    break;
+                }
+                __nanosleep(polls < 64u ? 40u : 400u);
+                continue;
+            }
+            const uint32_t mine = ((needed >> lane) & 1u) ? (uint32_t)st : 0u;
+            excl += warp_sum(mine);
+            if (first < 32) break;
+            look -= 32;
+        }
+    }
+    if (lane == 0) {
+        if (ok) {
+            if (tile > 0) atomicExch(&sc.tile_state[tile], kFlagInclusive | (excl + total));
+        } else {
+            atomicCAS(sc.status, 0, -5 /* SAPS_ERR_TIMEOUT */);
+        }
+    }
+    *out_excl = excl;
+    return ok;
+}
+
 template <bool GATHER>
 __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
 {
@@ -72,52 +124,15 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
         total += c;
     }
 
-    // ---- order the tiles: decoupled look-back, done by warp 0 ----
+    // ---- order the tiles ----
     if (warp == 0) {
-        if (lane == 0)
-            atomicExch(&a.scratch.tile_state[tile],
-                       (tile == 0 ? kFlagInclusive : kFlagAggregate) | total);
-        uint32_t excl = 0;
-        bool ok = true;
-        if (tile > 0) {
-            long long look = (long long)tile - 1;  // newest tile of the window
-            uint32_t polls = 0;
-            while (true) {
-                const long long idx = look - lane;
-                // tiles before the first count as "inclusive prefix 0"
-                const unsigned long long st =
-                    idx >= 0 ? peek_state(&a.scratch.tile_state[idx]) : kFlagInclusive;
-                const uint32_t flag = (uint32_t)(st >> 32);
-                const uint32_t incl = __ballot_sync(0xFFFFFFFFu, flag == 2u);
-                const uint32_t empty = __ballot_sync(0xFFFFFFFFu, flag == 0u);
-                const int first = incl ? (__ffs(incl) - 1) : 32;  // nearest inclusive prefix
-                const uint32_t needed = first >= 31 ? 0xFFFFFFFFu : ((2u << first) - 1u);
-                if (empty & needed) {
-                    // a predecessor has not published yet: back off and poll again
-                    ++polls;
-                    bool give_up = polls > a.spin_limit;
-                    if ((polls & 63u) == 0u)
-                        give_up |= *reinterpret_cast<volatile int*>(a.scratch.status) != 0;
-                    if (__any_sync(0xFFFFFFFFu, give_up)) {
-                        ok = false;
-                        break;
-                    }
-                    __nanosleep(polls < 64u ? 40u : 400u);
-                    continue;
-                }
-                const uint32_t mine = ((needed >> lane) & 1u) ? (uint32_t)st : 0u;
-                excl += warp_sum(mine);
-                if (first < 32) break;
-                look -= 32;
-            }
-        }
+        uint32_t excl;
+        const bool ok = lookback_exclusive(a.scratch, tile, total, a.spin_limit, lane, &excl);
         if (lane == 0) {
             if (ok) {
-                if (tile > 0) atomicExch(&a.scratch.tile_state[tile], kFlagInclusive | (excl + total));
                 a.scratch.tile_excl[tile] = excl;
                 s_excl = excl;
             } else {
-                atomicCAS(a.scratch.status, 0, -5 /* SAPS_ERR_TIMEOUT */);
                 s_abort = 1;
             }
         }
@@ -150,11 +165,86 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
         if (total == 0) return;
         const uint32_t room = base < a.cap ? a.cap - base : 0u;
         const uint32_t take = total < room ? total : room;
-        for (uint32_t i = 0; i < (uint32_t)a.n; ++i) {
-            const float* __restrict__ row = a.x + (size_t)i * a.ld;
-            float* __restrict__ out = a.out_vals + (size_t)i * a.cap + base;
-            for (uint32_t q = tid; q < take; q += kThreads) out[q] = __ldg(row + s_kept[q]);
+        // one flat loop over (worker, kept column): with a sparse mask a tile keeps only a few
+        // columns, so looping over workers inside keeps every thread busy and all the
+        // (uncoalesced, sector-sized) loads of a tile in flight at once
+        const uint32_t items = (uint32_t)a.n * take;
+        for (uint32_t e = tid; e < items; e += kThreads) {
+            const uint32_t i = e / take, q = e - i * take;
+            a.out_vals[(size_t)i * a.cap + base + q] = __ldg(a.x + (size_t)i * a.ld + s_kept[q]);
         }
+    }
+}
+
+// Mask scan without model data (indices, count, per-tile prefixes for the fused emission).
+// One block covers kScanSub column tiles, one warp each, so that the look-back chain has
+// eight times fewer links than tiles.
+constexpr int kScanSub = kThreads / 32;
+
+__global__ void __launch_bounds__(kThreads) scan_kernel(const PackArgs a)
+{
+    constexpr int kWords = kTileCols / 32;  // mask words per tile
+    __shared__ uint32_t s_big, s_excl, s_abort;
+    __shared__ uint32_t s_cnt[kScanSub];
+    __shared__ uint32_t s_word[kScanSub][kWords];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        s_big = atomicAdd(a.scratch.ticket, 1u);
+        s_abort = 0;
+    }
+    __syncthreads();
+    const uint32_t big = s_big;
+    const uint32_t nbig = (a.scratch.ntiles + kScanSub - 1) / kScanSub;
+    if (big >= nbig) return;
+    const uint32_t tile = big * kScanSub + warp;            // this warp's tile (may lie past the end)
+    const uint64_t col0 = (uint64_t)tile * kTileCols;
+
+    uint32_t cnt = 0;
+    for (int s = 0; s < kWords; ++s) {
+        const uint64_t k = col0 + s * 32 + lane;
+        const bool kept = (k < a.N) && column_kept(a.col_offset + (uint32_t)k, a.key);
+        const uint32_t w = __ballot_sync(0xFFFFFFFFu, kept);
+        if (lane == 0) s_word[warp][s] = w;
+        cnt += __popc(w);
+    }
+    if (lane == 0) s_cnt[warp] = cnt;
+    __syncthreads();
+    uint32_t before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < kScanSub; ++w) {
+        const uint32_t c = s_cnt[w];
+        before += (w < warp) ? c : 0u;
+        total += c;
+    }
+    if (warp == 0) {
+        uint32_t excl;
+        const bool ok = lookback_exclusive(a.scratch, big, total, a.spin_limit, lane, &excl);
+        if (lane == 0) {
+            s_excl = excl;
+            if (!ok) s_abort = 1;
+        }
+    }
+    __syncthreads();
+    if (s_abort) return;
+    const uint32_t base = s_excl + before;
+    if (tile < a.scratch.ntiles) {
+        if (lane == 0) a.scratch.tile_excl[tile] = base;
+        if (a.out_idx != nullptr) {
+            uint32_t r = base;
+            for (int s = 0; s < kWords; ++s) {
+                const uint32_t w = s_word[warp][s];
+                if ((w >> lane) & 1u) {
+                    const uint32_t mine = r + __popc(w & ((1u << lane) - 1u));
+                    if (mine < a.cap) a.out_idx[mine] = a.col_offset + (uint32_t)(col0 + s * 32 + lane);
+                }
+                r += __popc(w);
+            }
+        }
+    }
+    if (big == nbig - 1 && tid == 0) {
+        if (a.out_count != nullptr) *a.out_count = s_excl + total;
+        if (s_excl + total > a.cap) atomicCAS(a.scratch.status, 0, -4 /* SAPS_ERR_OVERFLOW */);
     }
 }
 
@@ -177,7 +267,7 @@ cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream)
     if (a.out_vals != nullptr)
         pack_kernel<true><<<ntiles, kThreads, 0, stream>>>(a);
     else
-        pack_kernel<false><<<ntiles, kThreads, 0, stream>>>(a);
+        scan_kernel<<<(ntiles + kScanSub - 1) / kScanSub, kThreads, 0, stream>>>(a);
     return cudaGetLastError();
 }
 
