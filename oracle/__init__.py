@@ -61,6 +61,12 @@ def _c():
         lib.orc_pair_average.argtypes = [i32, u64, vp, vp, vp]
         lib.orc_round.restype = None
         lib.orc_round.argtypes = [i32, u64, vp, vp, f32, vp, u64, u64, dbl, vp]
+        lib.orc_round_eq7.restype = None
+        lib.orc_round_eq7.argtypes = [i32, u64, vp, vp, f32, vp, u64, u64, dbl, vp]
+        lib.orc_unpack_avg.restype = None
+        lib.orc_unpack_avg.argtypes = [i32, u64, vp, vp, u64, vp, u64]
+        lib.orc_consensus_distance.restype = dbl
+        lib.orc_consensus_distance.argtypes = [i32, u64, vp]
         _lib = lib
     return _lib
 
@@ -151,6 +157,39 @@ def gossip_round(x: np.ndarray, g, lr: float, pairs, seed: int, t: int,
     _c().orc_round(n, N, _ptr(x), _ptr(g), float(lr), _ptr(p), seed, t, float(keep_frac),
                    _ptr(m))
     return m
+
+
+def gossip_round_eq7(x: np.ndarray, g, lr: float, pairs, seed: int, t: int,
+                     keep_frac: float) -> np.ndarray:
+    """One round in the order of Eq. 7 (average the current models, then subtract the
+    gradient step), in place on ``x``; returns the round's mask."""
+    _f32_matrix(x, "x", True)
+    n, N = x.shape
+    if g is not None:
+        _f32_matrix(g, "g")
+        assert g.shape == x.shape
+    p = np.ascontiguousarray(pairs, dtype=np.int32)
+    _check_pairs(p, n)
+    m = np.empty(N, dtype=np.uint8)
+    _c().orc_round_eq7(n, N, _ptr(x), _ptr(g), float(lr), _ptr(p), seed, t, float(keep_frac),
+                       _ptr(m))
+    return m
+
+
+def unpack_avg(x: np.ndarray, recv: np.ndarray, idx: np.ndarray, count: int) -> None:
+    """In place: x[i, idx[r]] = (x[i, idx[r]] + recv[i, r]) / 2 for r < count."""
+    _f32_matrix(x, "x", True)
+    _f32_matrix(recv, "recv")
+    assert recv.shape[0] == x.shape[0] and idx.dtype == np.uint32 and idx.flags.c_contiguous
+    assert count <= idx.shape[0]
+    _c().orc_unpack_avg(x.shape[0], x.shape[1], _ptr(x), _ptr(recv), recv.shape[1], _ptr(idx),
+                        int(count))
+
+
+def consensus_distance(x: np.ndarray) -> float:
+    """|| X - mean over workers ||_F^2 in double precision."""
+    _f32_matrix(x, "x")
+    return float(_c().orc_consensus_distance(x.shape[0], x.shape[1], _ptr(x)))
 
 
 def _check_pairs(p: np.ndarray, n: int) -> None:

@@ -172,3 +172,47 @@ void orc_round(int n, uint64_t N, float *x, const float *g, float lr, const int3
     orc_mask(seed, t, keep_frac, N, m);
     orc_pair_average(n, N, x, pairs, m);
 }
+
+/* ---- variants and companions of the round ------------------------------------ */
+
+/* The update in the order of Eq. 7 (the form the convergence analysis uses):
+ * X_{t+1} = X_t o not M_t + (X_t o M_t) W_t - gamma G(X_t).  The kept coordinates of the
+ * CURRENT models are averaged first, then every worker subtracts its own gradient step. */
+void orc_round_eq7(int n, uint64_t N, float *x, const float *g, float lr, const int32_t *pairs,
+                   uint64_t seed, uint64_t t, double keep_frac, uint8_t *m)
+{
+    orc_mask(seed, t, keep_frac, N, m);
+    orc_pair_average(n, N, x, pairs, m);
+    orc_sgd(n, N, x, g, lr);
+}
+
+/* Receiving side of the exchange (Algorithm 2, merge): worker i holds its own model x_i and
+ * the buffer recv[i*cap + r] it received, whose r-th entry belongs to column idx[r]; the kept
+ * coordinates become the mean of the local and the received value. */
+void orc_unpack_avg(int n, uint64_t N, float *x, const float *recv, uint64_t cap,
+                    const uint32_t *idx, uint64_t count)
+{
+    for (int i = 0; i < n; ++i)
+        for (uint64_t r = 0; r < count && r < cap; ++r) {
+            float s = x[(size_t)i * N + idx[r]] + recv[(size_t)i * cap + r];
+            x[(size_t)i * N + idx[r]] = 0.5f * s;
+        }
+}
+
+/* Consensus distance of Theorem 1 / Lemma 2: || X - Xbar 1^T ||_F^2, the sum over all
+ * coordinates of the squared deviations of the n workers from their mean.  fp64. */
+double orc_consensus_distance(int n, uint64_t N, const float *x)
+{
+    double total = 0.0;
+    for (uint64_t k = 0; k < N; ++k) {
+        double mean = 0.0;
+        for (int i = 0; i < n; ++i)
+            mean += (double)x[(size_t)i * N + k];
+        mean /= (double)n;
+        for (int i = 0; i < n; ++i) {
+            double d = (double)x[(size_t)i * N + k] - mean;
+            total += d * d;
+        }
+    }
+    return total;
+}

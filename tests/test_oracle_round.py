@@ -221,3 +221,99 @@ def test_rejects_bad_pairs():
         oracle.gossip_round(x, None, 0.0, [1, 2, 0, 3], 0, 1, 0.5)
     with pytest.raises(ValueError):
         oracle.gossip_round(x, None, 0.0, [1, 0, 4, 2], 0, 1, 0.5)
+
+
+# ---- Eq. 7 ordering, receiving side, consensus distance ---------------------------------------
+
+def test_eq7_order_is_the_matrix_form():
+    # X' = X o not M + (X o M) W - gamma G, evaluated densely in double precision
+    n, N, lr, p = 8, 4001, 0.05, 0.3
+    x, g = _inputs(n, N, seed=12)
+    pairs = synth.random_perfect_matching(n, synth.matching_rng(12))
+    W = ps.generate_W(list(pairs))
+    m = oracle.mask(4, 6, p, N).astype(np.float64)
+    X, G = x.astype(np.float64), g.astype(np.float64)
+    want = X * (1 - m)[None, :] + W @ (X * m[None, :]) - np.float64(np.float32(lr)) * G
+    got = x.copy()
+    m2 = oracle.gossip_round_eq7(got, g, lr, pairs, 4, 6, p)
+    assert (m2 == m).all()
+    # three fp32 roundings (sum, product lr*g, difference) against the exact value
+    tol = 2.0 ** -23 * (np.abs(want) + np.abs(X) + np.abs(lr * G)) + 1e-45
+    assert (np.abs(got.astype(np.float64) - want) <= tol).all()
+    # and it is NOT the Algorithm 2 order: there the gradient step is averaged too
+    alg2 = x.copy()
+    oracle.gossip_round(alg2, g, lr, pairs, 4, 6, p)
+    kept = m.astype(bool)
+    assert (alg2[:, ~kept] == got[:, ~kept]).all()
+    assert not np.array_equal(alg2[:, kept], got[:, kept])
+    diff = got.astype(np.float64) - alg2.astype(np.float64)
+    # difference on kept coordinates = -lr (g_i - (g_i + g_j)/2) up to rounding
+    want_diff = -lr * (G - W @ G)
+    assert np.allclose(diff[:, kept], want_diff[:, kept], rtol=0, atol=1e-6)
+
+
+def test_eq7_order_reductions():
+    n, N = 6, 3001
+    x, g = _inputs(n, N, seed=13)
+    pairs = [1, 0, 3, 2, 5, 4]
+    # without a gradient the two orders coincide bit for bit
+    a, b = x.copy(), x.copy()
+    oracle.gossip_round(a, None, 0.0, pairs, 1, 2, 0.4)
+    oracle.gossip_round_eq7(b, None, 0.0, pairs, 1, 2, 0.4)
+    assert (a.view(np.uint32) == b.view(np.uint32)).all()
+    # empty mask: plain SGD in both orders
+    a, b = x.copy(), x.copy()
+    oracle.gossip_round(a, g, 0.1, pairs, 1, 2, 0.0)
+    oracle.gossip_round_eq7(b, g, 0.1, pairs, 1, 2, 0.0)
+    assert (a == b).all() and (a == x - np.float32(0.1) * g).all()
+    # column sums move by exactly the summed gradient step (W is doubly stochastic)
+    c = x.copy()
+    oracle.gossip_round_eq7(c, g, 0.1, pairs, 1, 2, 0.5)
+    want = x.astype(np.float64).sum(0) - 0.1 * g.astype(np.float64).sum(0)
+    assert np.allclose(c.astype(np.float64).sum(0), want, rtol=0, atol=1e-5)
+
+
+def test_unpack_avg_is_the_receiving_side_of_the_round():
+    n, N = 6, 7001
+    x, g = _inputs(n, N, seed=14)
+    pairs = [3, 2, 1, 0, 5, 4]
+    a = x.copy()
+    oracle.sgd(a, g, 0.05)
+    m = oracle.mask(6, 4, 0.15, N)
+    vals, idx, count = oracle.pack(a, m)
+    recv = np.ascontiguousarray(vals[pairs])             # what each worker gets from its peer
+    oracle.unpack_avg(a, recv, idx, count)
+    oracle.gossip_round(x, g, 0.05, pairs, 6, 4, 0.15)
+    assert (x.view(np.uint32) == a.view(np.uint32)).all()
+    # hand-checkable: one worker, two kept columns
+    y = np.array([[1.0, 2.0, 3.0, 4.0]], np.float32)
+    oracle.unpack_avg(y, np.array([[10.0, 20.0]], np.float32), np.array([1, 3], np.uint32), 2)
+    assert (y == np.array([[1.0, 6.0, 3.0, 12.0]], np.float32)).all()
+    # count smaller than the buffer: the rest is ignored
+    y = np.array([[1.0, 2.0, 3.0, 4.0]], np.float32)
+    oracle.unpack_avg(y, np.array([[10.0, 20.0]], np.float32), np.array([1, 3], np.uint32), 1)
+    assert (y == np.array([[1.0, 6.0, 3.0, 4.0]], np.float32)).all()
+
+
+def test_consensus_distance_closed_forms():
+    rng = np.random.default_rng(5)
+    a = rng.standard_normal(1000).astype(np.float32)
+    # identical workers: zero; two opposite workers: 2 sum a^2
+    assert oracle.consensus_distance(np.stack([a, a, a])) == 0.0
+    assert np.isclose(oracle.consensus_distance(np.stack([a, -a])), 2 * (a.astype(np.float64) ** 2).sum(),
+                      rtol=1e-14)
+    # n * (population variance over workers), summed over coordinates: a library routine
+    x, _ = _inputs(16, 5000, seed=15)
+    want = 16 * np.var(x.astype(np.float64), axis=0).sum()
+    assert np.isclose(oracle.consensus_distance(x), want, rtol=1e-12)
+    # adding the same vector to every worker changes nothing (up to the fp32 rounding of the inputs)
+    shifted = (x.astype(np.float64) + 3.0).astype(np.float32)
+    assert np.isclose(oracle.consensus_distance(shifted), want, rtol=1e-5)
+    # hand-checkable: workers (0, 2) and (4, 6): means 2 and 4, deviations +-2 -> 4 * 4
+    assert oracle.consensus_distance(np.array([[0.0, 2.0], [4.0, 6.0]], np.float32)) == 16.0
+    # full gossip with a connected schedule drives it to (numerically) zero
+    y, _ = _inputs(8, 500, seed=16)
+    d0 = oracle.consensus_distance(y)
+    for r in range(3):
+        oracle.gossip_round(y, None, 0.0, synth.hypercube_pairs(8, r), 0, r + 1, 1.0)
+    assert oracle.consensus_distance(y) == 0.0 < d0
