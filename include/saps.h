@@ -121,6 +121,18 @@ SAPS_API int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, 
                     uint64_t t, double keep_frac, float* out_vals, uint32_t* out_idx,
                     uint32_t* out_count, void* stream);
 
+/* Order of the two halves of the update.
+ *   SAPS_ORDER_SGD_FIRST     Algorithm 2 (default): a = x - lr g, then the kept coordinates of
+ *                            a matched pair become the mean of the two a's.
+ *   SAPS_ORDER_GOSSIP_FIRST  Eq. 7, the form the convergence analysis uses:
+ *                            X' = X o not M + (X o M) W - lr G(X): the kept coordinates of the
+ *                            CURRENT models are averaged, then each worker subtracts its own
+ *                            gradient step.  The emitted wire buffer then holds x (not a).
+ * A per-round learning rate (gamma_t of Eq. 7) is simply the lr argument of each call. */
+#define SAPS_ORDER_SGD_FIRST    0
+#define SAPS_ORDER_GOSSIP_FIRST 1
+SAPS_API int saps_set_update_order(saps_ctx* ctx, int order);
+
 /* ---- pack (Eq. 2; "sends the non-zero elements", Section II-B) -------------------------- */
 
 /* Slots per worker that out_vals / out_idx must hold for this keep_frac:
@@ -144,6 +156,19 @@ SAPS_API int saps_set_pack_capacity(saps_ctx* ctx, uint64_t cap);
  * word is set to SAPS_ERR_OVERFLOW.  Slots r >= count are not written. */
 SAPS_API int saps_pack(saps_ctx* ctx, const float* x, uint64_t t, double keep_frac, float* out_vals,
               uint32_t* out_idx, uint32_t* out_count, void* stream);
+
+/* Receiving side of the exchange (Algorithm 2: ExchangeModelWithPeer and the merge), for a
+ * deployment where the packed buffers really travel: every worker i averages its kept
+ * coordinates with the buffer it received,
+ *     x[i][idx[r]] = 1/2 (x[i][idx[r]] + recv_vals[src(i)][r]),  r < *count,
+ * where src(i) = pairs[i] when pairs (host, n entries) is given - recv_vals is then simply
+ * the senders' buffer [n, cap] as saps_pack wrote it, and a worker without a peer is left
+ * alone - or src(i) = i when pairs is NULL (recv_vals already holds, in row i, what worker i
+ * received).  idx, count: device, as written by saps_pack; cap = saps_pack_capacity(ctx,
+ * keep_frac).  SGD-only round + saps_pack + saps_unpack_avg equals saps_round bit for bit. */
+SAPS_API int saps_unpack_avg(saps_ctx* ctx, float* x, const float* recv_vals, const uint32_t* idx,
+                             const uint32_t* count, double keep_frac, const int32_t* pairs,
+                             void* stream);
 
 /* saps_pack for callers that must not allocate device memory.  (The paper has no counterpart:
  * this entry point exists for integration only.)
@@ -209,9 +234,10 @@ SAPS_API int saps_set_select_state(saps_ctx* ctx, const int64_t* R, uint64_t las
  *   pairs_list != NULL : pairs_list[r*n .. r*n+n-1] (host, T x n), else
  *   bandwidth  != NULL : saps_select_peers(ctx, bandwidth, t) (runs on the host ahead of
  *                        the GPU; it never depends on device data).
- * out_pairs_log (host, T x n) receives the matchings used, or may be NULL. */
+ * out_pairs_log (host, T x n) receives the matchings used, or may be NULL.
+ * lr_list (host, T floats) gives a learning rate per round (gamma_t), or NULL to use lr. */
 SAPS_API int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t t_first,
-                    uint64_t T, double keep_frac, const int32_t* pairs_list,
+                    uint64_t T, double keep_frac, const float* lr_list, const int32_t* pairs_list,
                     const double* bandwidth, int32_t* out_pairs_log, void* stream);
 
 /* ---- host-buffer entry point ----------------------------------------------------------------- */
@@ -234,6 +260,23 @@ SAPS_API int saps_round_pack_host(saps_ctx* ctx, float* x_host, const float* g_h
                                   uint32_t* out_count_host, float* d_vals, uint32_t* d_idx,
                                   uint32_t* d_count);
 
+/* ---- consensus and communication metrics -------------------------------------------------------- */
+
+/* Consensus distance of Theorem 1 / Lemma 2: *out = || X - Xbar 1^T ||_F^2, the sum over all
+ * coordinates of the squared deviations of the n workers from their mean, accumulated in
+ * fp64 in a fixed order (the result is reproducible).  x: device [n, ld]; out: device, one
+ * double.  Reads x once.  The first call allocates ceil(N/2048) doubles of scratch. */
+SAPS_API int saps_consensus_distance(saps_ctx* ctx, const float* x, double* out, void* stream);
+
+/* Host only.  Communication figures of one round (Table 1; the bandwidth utilisation of
+ * Section IV-D is the bottleneck bandwidth of the chosen pairs): out5[0] = values a matched
+ * worker sends + receives (2 count), out5[1] = the same in bytes, out5[2] = smallest and
+ * out5[3] = mean symmetrised bandwidth over the chosen pairs, out5[4] = time in seconds to
+ * move one buffer over the slowest chosen link, 32 count / (out5[2] * bits_per_s_per_unit)
+ * (bits_per_s_per_unit = 1e6 when the matrix is in Mb/s). */
+SAPS_API int saps_comm_stats(const saps_ctx* ctx, const double* bandwidth, const int32_t* pairs,
+                             uint64_t count, double bits_per_s_per_unit, double* out5);
+
 /* ---- measurement ------------------------------------------------------------------------------- */
 
 /* Optional cudaEvent_t pair (as void*; NULL, NULL switches it off).  When set, saps_round
@@ -241,6 +284,12 @@ SAPS_API int saps_round_pack_host(saps_ctx* ctx, float* x_host, const float* g_h
  * just behind it, on the call's stream, so that a benchmark can time that one kernel inside
  * a longer step.  The events stay owned by the caller. */
 SAPS_API int saps_set_timing_events(saps_ctx* ctx, void* before, void* after);
+
+/* Test hook for the bounded wait of the compaction scan: look-back tile `skip_tile` never
+ * publishes its state, so its successors run out of polls after `spin_limit` tries (0 = the
+ * default budget) and the kernel ends with SAPS_ERR_TIMEOUT in the status word instead of
+ * hanging.  skip_tile = 0xFFFFFFFF switches the hook off.  Nothing faults or traps. */
+SAPS_API int saps_debug_inject(saps_ctx* ctx, uint32_t skip_tile, uint32_t spin_limit);
 
 /* ---- errors ----------------------------------------------------------------------------------- */
 

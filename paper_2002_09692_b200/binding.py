@@ -59,7 +59,12 @@ _SIGNATURES = {
     "saps_select_reset": (_i32, [_vp]),
     "saps_get_select_state": (_i32, [_vp, _vp, ctypes.POINTER(_u64)]),
     "saps_set_select_state": (_i32, [_vp, _vp, _u64]),
-    "saps_run_rounds": (_i32, [_vp, _vp, _vp, _f32, _u64, _u64, _f64, _vp, _vp, _vp, _vp]),
+    "saps_run_rounds": (_i32, [_vp, _vp, _vp, _f32, _u64, _u64, _f64, _vp, _vp, _vp, _vp, _vp]),
+    "saps_set_update_order": (_i32, [_vp, _i32]),
+    "saps_unpack_avg": (_i32, [_vp, _vp, _vp, _vp, _vp, _f64, _vp, _vp]),
+    "saps_consensus_distance": (_i32, [_vp, _vp, _vp, _vp]),
+    "saps_comm_stats": (_i32, [_vp, _vp, _vp, _u64, _f64, _vp]),
+    "saps_debug_inject": (_i32, [_vp, _u32, _u32]),
     "saps_round_host": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp, _vp]),
     "saps_round_pack_host": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "saps_set_timing_events": (_i32, [_vp, _vp, _vp]),
@@ -221,11 +226,43 @@ def saps_set_select_state(ctx, R, last_t: int) -> None:
 
 
 def saps_run_rounds(ctx, x, g, lr, t_first, T, keep_frac, pairs_list=None, bandwidth=None,
-                    out_pairs_log=None, stream=None) -> None:
+                    out_pairs_log=None, stream=None, lr_list=None) -> None:
     """pairs_list: T x n int32 numpy array or None; bandwidth: n x n float64 numpy array or
-    None; out_pairs_log: T x n int32 numpy array to fill, or None."""
-    _check(_lib.saps_run_rounds(ctx, _ptr(x), _ptr(g), lr, t_first, T, keep_frac, _ptr(pairs_list),
-                                _ptr(bandwidth), _ptr(out_pairs_log), _stream(stream)), "saps_run_rounds")
+    None; out_pairs_log: T x n int32 numpy array to fill, or None; lr_list: T float32 numpy
+    array (a learning rate per round) or None."""
+    _check(_lib.saps_run_rounds(ctx, _ptr(x), _ptr(g), lr, t_first, T, keep_frac, _ptr(lr_list),
+                                _ptr(pairs_list), _ptr(bandwidth), _ptr(out_pairs_log), _stream(stream)),
+           "saps_run_rounds")
+
+
+SAPS_ORDER_SGD_FIRST = 0
+SAPS_ORDER_GOSSIP_FIRST = 1
+
+
+def saps_set_update_order(ctx, order: int) -> None:
+    _check(_lib.saps_set_update_order(ctx, order), "saps_set_update_order")
+
+
+def saps_unpack_avg(ctx, x, recv_vals, idx, count, keep_frac, pairs=None, stream=None) -> None:
+    _check(_lib.saps_unpack_avg(ctx, _ptr(x), _ptr(recv_vals), _ptr(idx), _ptr(count), keep_frac,
+                                None if pairs is None else _pairs(pairs), _stream(stream)), "saps_unpack_avg")
+
+
+def saps_consensus_distance(ctx, x, out, stream=None) -> None:
+    _check(_lib.saps_consensus_distance(ctx, _ptr(x), _ptr(out), _stream(stream)), "saps_consensus_distance")
+
+
+def saps_comm_stats(ctx, bandwidth, pairs, count: int, bits_per_s_per_unit: float = 1e6):
+    """bandwidth: n x n float64 numpy array.  Returns a dict of the five figures."""
+    out = (ctypes.c_double * 5)()
+    _check(_lib.saps_comm_stats(ctx, _ptr(bandwidth), _pairs(pairs), count, bits_per_s_per_unit, out),
+           "saps_comm_stats")
+    keys = ("values_per_worker", "bytes_per_worker", "bottleneck_bandwidth", "mean_bandwidth", "comm_time_s")
+    return dict(zip(keys, out))
+
+
+def saps_debug_inject(ctx, skip_tile: int, spin_limit: int) -> None:
+    _check(_lib.saps_debug_inject(ctx, skip_tile, spin_limit), "saps_debug_inject")
 
 
 def saps_round_host(ctx, x_host, g_host, lr, pairs, t, keep_frac, d_x, d_g) -> None:

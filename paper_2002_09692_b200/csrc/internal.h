@@ -74,6 +74,7 @@ struct RoundArgs {
     uint32_t col_offset;   // global index of this shard's column 0 (mask hash input)
     uint32_t tile_begin;   // first column tile to process
     uint32_t tile_count;   // number of column tiles to process
+    int gossip_first;      // 0: Algorithm 2's order (SGD, then average); 1: Eq. 7's order
     // emission of the wire buffer (all NULL/0 when not emitting)
     float* out_vals;
     uint32_t cap;
@@ -95,12 +96,32 @@ struct PackArgs {
     uint32_t* out_count;  // may be NULL
     ScratchView scratch;
     uint32_t spin_limit;
+    uint32_t skip_tile;   // test hook: this look-back tile never publishes (0xFFFFFFFF = none)
 };
 
 cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream);
 
 cudaError_t launch_mask(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t* out_bits,
                         cudaStream_t stream);
+
+// Receiving side of the exchange: x[i][idx[r]] = (x[i][idx[r]] + recv[src[i]][r]) / 2.
+struct UnpackArgs {
+    float* x;
+    size_t ld;
+    int n;
+    const float* recv;     // [n, cap]
+    uint32_t cap;
+    const uint32_t* idx;   // global columns
+    const uint32_t* count; // device
+    uint32_t col_offset;
+    uint32_t N;
+    uint8_t src[kMaxWorkers];  // row of recv that worker i received, kNoPeer = nothing received
+};
+cudaError_t launch_unpack_avg(const UnpackArgs& a, cudaStream_t stream);
+
+// || X - mean over workers ||_F^2: per-tile partial sums, then one block adds them in order.
+cudaError_t launch_consensus(const float* x, size_t ld, uint32_t N, int n, uint32_t ntiles,
+                             double* partials, double* out, cudaStream_t stream);
 
 // Compaction on the library's static scratch area (no allocation anywhere on the path).
 constexpr uint32_t kStaticMaxTiles = 65536;  // kTileCols columns each: N <= 134,217,728

@@ -38,9 +38,11 @@ __device__ __forceinline__ uint32_t warp_sum(uint32_t v)
 // Returns false when a predecessor did not publish within the poll budget (or another tile
 // already reported an error); the status word then holds SAPS_ERR_TIMEOUT.
 __device__ __forceinline__ bool lookback_exclusive(const ScratchView& sc, uint32_t tile, uint32_t total,
-                                                   uint32_t spin_limit, int lane, uint32_t* out_excl)
+                                                   uint32_t spin_limit, uint32_t skip_tile, int lane,
+                                                   uint32_t* out_excl)
 {
-    if (lane == 0)
+    const bool publish = tile != skip_tile;  // the test hook makes one tile stay silent
+    if (lane == 0 && publish)
         atomicExch(&sc.tile_state[tile], (tile == 0 ? kFlagInclusive : kFlagAggregate) | total);
     uint32_t excl = 0;
     bool ok = true;
@@ -76,7 +78,7 @@ __device__ __forceinline__ bool lookback_exclusive(const ScratchView& sc, uint32
     }
     if (lane == 0) {
         if (ok) {
-            if (tile > 0) atomicExch(&sc.tile_state[tile], kFlagInclusive | (excl + total));
+            if (tile > 0 && publish) atomicExch(&sc.tile_state[tile], kFlagInclusive | (excl + total));
         } else {
             atomicCAS(sc.status, 0, -5 /* SAPS_ERR_TIMEOUT */);
         }
@@ -127,7 +129,7 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
     // ---- order the tiles ----
     if (warp == 0) {
         uint32_t excl;
-        const bool ok = lookback_exclusive(a.scratch, tile, total, a.spin_limit, lane, &excl);
+        const bool ok = lookback_exclusive(a.scratch, tile, total, a.spin_limit, a.skip_tile, lane, &excl);
         if (lane == 0) {
             if (ok) {
                 a.scratch.tile_excl[tile] = excl;
@@ -219,7 +221,7 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const PackArgs a)
     }
     if (warp == 0) {
         uint32_t excl;
-        const bool ok = lookback_exclusive(a.scratch, big, total, a.spin_limit, lane, &excl);
+        const bool ok = lookback_exclusive(a.scratch, big, total, a.spin_limit, a.skip_tile, lane, &excl);
         if (lane == 0) {
             s_excl = excl;
             if (!ok) s_abort = 1;
@@ -257,7 +259,90 @@ __global__ void __launch_bounds__(kThreads) mask_kernel(uint32_t N, uint32_t col
     if ((threadIdx.x & 31) == 0 && k < N) out_bits[k >> 5] = w;
 }
 
+// Receiving side of the exchange (Algorithm 2, merge): one thread per (worker, received entry).
+__global__ void __launch_bounds__(kThreads) unpack_avg_kernel(const UnpackArgs a)
+{
+    const uint32_t src = a.src[blockIdx.y];
+    if (src == kNoPeer) return;
+    uint32_t count = *a.count;
+    if (count > a.cap) count = a.cap;
+    const uint32_t r = blockIdx.x * kThreads + threadIdx.x;
+    if (r >= count) return;
+    const uint32_t k = __ldg(a.idx + r) - a.col_offset;
+    if (k >= a.N) return;  // an index list of another shard: stay in bounds
+    float* p = a.x + (size_t)blockIdx.y * a.ld + k;
+    *p = __fmul_rn(0.5f, __fadd_rn(*p, __ldg(a.recv + (size_t)src * a.cap + r)));
+}
+
+// Consensus distance, one block per column tile.  Per column the deviations are taken from
+// worker 0's value (exact in fp64), sum d^2 - (sum d)^2 / n, so that identical workers give
+// exactly zero and nearly identical ones lose no digits.
+__global__ void __launch_bounds__(kThreads) consensus_partial_kernel(const float* __restrict__ x, size_t ld,
+                                                                     uint32_t N, int n, double* partials)
+{
+    __shared__ double s_part[kThreads / 32];
+    const int tid = threadIdx.x;
+    double acc = 0.0;
+    const uint64_t col0 = (uint64_t)blockIdx.x * kTileCols;
+#pragma unroll 2
+    for (int u = 0; u < kTileCols / kThreads; ++u) {
+        const uint64_t k = col0 + (uint64_t)u * kThreads + tid;
+        if (k < N) {
+            const double pivot = (double)__ldcs(x + k);
+            double sd = 0.0, sdd = 0.0;
+            for (int i = 1; i < n; ++i) {
+                const double d = (double)__ldcs(x + (size_t)i * ld + k) - pivot;
+                sd += d;
+                sdd += d * d;
+            }
+            acc += sdd - sd * sd / (double)n;
+        }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, d);
+    if ((tid & 31) == 0) s_part[tid >> 5] = acc;
+    __syncthreads();
+    if (tid == 0) {
+        double t = 0.0;
+        for (int w = 0; w < kThreads / 32; ++w) t += s_part[w];
+        partials[blockIdx.x] = t;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) consensus_final_kernel(const double* partials, uint32_t count,
+                                                                   double* out)
+{
+    __shared__ double s_part[kThreads];
+    double acc = 0.0;
+    for (uint32_t i = threadIdx.x; i < count; i += kThreads) acc += partials[i];
+    s_part[threadIdx.x] = acc;
+    __syncthreads();
+    for (int d = kThreads / 2; d > 0; d >>= 1) {
+        if ((int)threadIdx.x < d) s_part[threadIdx.x] += s_part[threadIdx.x + d];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *out = s_part[0] < 0.0 ? 0.0 : s_part[0];
+}
+
 }  // namespace
+
+cudaError_t launch_unpack_avg(const UnpackArgs& a, cudaStream_t stream)
+{
+    if (a.cap == 0 || a.n == 0) return cudaSuccess;
+    dim3 grid((a.cap + kThreads - 1) / kThreads, a.n, 1);
+    unpack_avg_kernel<<<grid, kThreads, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_consensus(const float* x, size_t ld, uint32_t N, int n, uint32_t ntiles, double* partials,
+                             double* out, cudaStream_t stream)
+{
+    consensus_partial_kernel<<<ntiles, kThreads, 0, stream>>>(x, ld, N, n, partials);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    consensus_final_kernel<<<1, kThreads, 0, stream>>>(partials, ntiles, out);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream)
 {

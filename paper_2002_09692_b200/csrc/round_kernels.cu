@@ -61,7 +61,9 @@ __device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t v, int lane)
     return v;
 }
 
-template <int VEC, bool HAS_G, bool EMIT>
+// GOSSIP_FIRST selects the order of Eq. 7 (average the current models, then subtract the
+// gradient step) instead of Algorithm 2's (SGD step first, then average).
+template <int VEC, bool HAS_G, bool EMIT, bool GOSSIP_FIRST>
 __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
 {
     constexpr int U = kTileCols / (kThreads * VEC);
@@ -109,7 +111,7 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
 #pragma unroll
             for (int c = 0; c < VEC; ++c)
                 bits[u] |= (column_kept(a.col_offset + col[u] + c, a.key) ? 1u : 0u) << c;
-            if (HAS_G) {
+            if (HAS_G && !GOSSIP_FIRST) {
 #pragma unroll
                 for (int c = 0; c < VEC; ++c) {
                     va[u].v[c] = sgd_step(va[u].v[c], wa[u].v[c], a.lr);
@@ -149,7 +151,7 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
             running += all;
         }
         total = running - excl;
-        // what each worker sends: its post-SGD value, before the average
+        // what each worker sends: its value before the average (post-SGD in Algorithm 2's order)
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             if (bits[u]) {
@@ -182,11 +184,22 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
                         }
                     }
                 }
+                if (HAS_G && GOSSIP_FIRST) {
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c) {
+                        va[u].v[c] = sgd_step(va[u].v[c], wa[u].v[c], a.lr);
+                        vb[u].v[c] = sgd_step(vb[u].v[c], wb[u].v[c], a.lr);
+                    }
+                }
                 if (HAS_G || bits[u]) {
                     store_stream<VEC>(xa + col[u], va[u]);
                     store_stream<VEC>(xb + col[u], vb[u]);
                 }
             } else if (HAS_G) {
+                if (GOSSIP_FIRST) {
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c) va[u].v[c] = sgd_step(va[u].v[c], wa[u].v[c], a.lr);
+                }
                 store_stream<VEC>(xa + col[u], va[u]);
             }
         }
@@ -198,10 +211,10 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
         if (ntail != 0 && tid < ntail && col_tile <= nfull && nfull < col_tile + kTileCols) {
             const uint32_t k = nfull + tid;
             float pa = xa[k], pb = 0.f;
-            if (HAS_G) pa = sgd_step(pa, ga[k], a.lr);
+            if (HAS_G && !GOSSIP_FIRST) pa = sgd_step(pa, ga[k], a.lr);
             if (paired) {
                 pb = xb[k];
-                if (HAS_G) pb = sgd_step(pb, gb[k], a.lr);
+                if (HAS_G && !GOSSIP_FIRST) pb = sgd_step(pb, gb[k], a.lr);
             }
             const bool kept = column_kept(a.col_offset + k, a.key);
             if constexpr (EMIT) {
@@ -214,8 +227,12 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
                     }
                 }
             }
+            if (paired && kept) pa = pb = pair_mean(pa, pb);
+            if (HAS_G && GOSSIP_FIRST) {
+                pa = sgd_step(pa, ga[k], a.lr);
+                if (paired) pb = sgd_step(pb, gb[k], a.lr);
+            }
             if (paired) {
-                if (kept) pa = pb = pair_mean(pa, pb);
                 if (HAS_G || kept) {
                     xa[k] = pa;
                     xb[k] = pb;
@@ -227,20 +244,25 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
     }
 }
 
-template <int VEC, bool HAS_G, bool EMIT>
+template <int VEC, bool HAS_G, bool EMIT, bool GOSSIP_FIRST>
 cudaError_t launch_variant(const RoundArgs& a, cudaStream_t stream)
 {
     dim3 grid(a.tile_count, a.groups.count, 1);
-    round_kernel<VEC, HAS_G, EMIT><<<grid, kThreads, 0, stream>>>(a);
+    round_kernel<VEC, HAS_G, EMIT, GOSSIP_FIRST><<<grid, kThreads, 0, stream>>>(a);
     return cudaGetLastError();
 }
 
 template <int VEC>
 cudaError_t launch_vec(const RoundArgs& a, bool emit, cudaStream_t stream)
 {
-    const bool has_g = a.g != nullptr;
-    if (has_g) return emit ? launch_variant<VEC, true, true>(a, stream) : launch_variant<VEC, true, false>(a, stream);
-    return emit ? launch_variant<VEC, false, true>(a, stream) : launch_variant<VEC, false, false>(a, stream);
+    if (a.g == nullptr)  // without a gradient both orders are the same update
+        return emit ? launch_variant<VEC, false, true, false>(a, stream)
+                    : launch_variant<VEC, false, false, false>(a, stream);
+    if (a.gossip_first)
+        return emit ? launch_variant<VEC, true, true, true>(a, stream)
+                    : launch_variant<VEC, true, false, true>(a, stream);
+    return emit ? launch_variant<VEC, true, true, false>(a, stream)
+                : launch_variant<VEC, true, false, false>(a, stream);
 }
 
 }  // namespace

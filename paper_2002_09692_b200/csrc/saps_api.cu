@@ -18,6 +18,10 @@ struct saps_ctx {
     uint32_t ntiles;
     uint64_t col_offset;    // global index of column 0 when this context holds a column shard
     cudaEvent_t ev_before, ev_after;  // optional: recorded around the round kernel
+    int gossip_first;       // update order: 0 Algorithm 2, 1 Eq. 7
+    uint32_t spin_limit;    // poll budget of the look-back
+    uint32_t skip_tile;     // test hook, 0xFFFFFFFF = off
+    double* partials;       // device, ntiles doubles, for the consensus distance
     uint64_t cap_override;  // 0 = capacity from the binomial bound
     // device scratch, allocated on first use on the then-current device
     void* scratch;
@@ -130,6 +134,7 @@ RoundArgs round_args(const saps_ctx* ctx, float* x, const float* g, float lr, co
     a.col_offset = (uint32_t)ctx->col_offset;
     a.tile_begin = 0;
     a.tile_count = ctx->ntiles;
+    a.gossip_first = ctx->gossip_first;
     a.out_vals = nullptr;
     a.cap = 0;
     a.tile_excl = nullptr;
@@ -172,6 +177,10 @@ int saps_create_ld(int n, uint64_t N, uint64_t ld, uint64_t seed, saps_ctx** out
     ctx->seed = seed;
     ctx->ntiles = (uint32_t)((N + kTileCols - 1) / kTileCols);
     ctx->cap_override = 0;
+    ctx->gossip_first = 0;
+    ctx->spin_limit = kSpinLimit;
+    ctx->skip_tile = 0xFFFFFFFFu;
+    ctx->partials = nullptr;
     ctx->ev_before = nullptr;
     ctx->ev_after = nullptr;
     ctx->col_offset = 0;
@@ -204,6 +213,7 @@ int saps_destroy(saps_ctx* ctx)
             cudaEventDestroy(ctx->lane_event[l]);
         }
     if (ctx->scratch != nullptr) cudaFree(ctx->scratch);
+    if (ctx->partials != nullptr) cudaFree(ctx->partials);
     delete ctx;
     return SAPS_OK;
 }
@@ -254,6 +264,89 @@ int saps_set_column_offset(saps_ctx* ctx, uint64_t col_offset)
     return SAPS_OK;
 }
 
+int saps_set_update_order(saps_ctx* ctx, int order)
+{
+    if (ctx == nullptr || (order != SAPS_ORDER_SGD_FIRST && order != SAPS_ORDER_GOSSIP_FIRST)) return SAPS_ERR_INVALID;
+    ctx->gossip_first = order == SAPS_ORDER_GOSSIP_FIRST;
+    return SAPS_OK;
+}
+
+int saps_unpack_avg(saps_ctx* ctx, float* x, const float* recv_vals, const uint32_t* idx, const uint32_t* count,
+                    double keep_frac, const int32_t* pairs, void* stream)
+{
+    if (ctx == nullptr || x == nullptr || recv_vals == nullptr || idx == nullptr || count == nullptr ||
+        !valid_frac(keep_frac))
+        return SAPS_ERR_INVALID;
+    UnpackArgs a;
+    if (pairs != nullptr) {
+        const int rc = check_pairs(ctx->n, pairs);
+        if (rc != SAPS_OK) return rc;
+    }
+    for (int i = 0; i < ctx->n; ++i)
+        a.src[i] = pairs == nullptr ? (uint8_t)i : (pairs[i] == i ? kNoPeer : (uint8_t)pairs[i]);
+    a.x = x;
+    a.ld = (size_t)ctx->ld;
+    a.n = ctx->n;
+    a.recv = recv_vals;
+    a.cap = (uint32_t)saps_pack_capacity(ctx, keep_frac);
+    a.idx = idx;
+    a.count = count;
+    a.col_offset = (uint32_t)ctx->col_offset;
+    a.N = (uint32_t)ctx->N;
+    return launch_unpack_avg(a, (cudaStream_t)stream) == cudaSuccess ? SAPS_OK : SAPS_ERR_CUDA;
+}
+
+int saps_consensus_distance(saps_ctx* ctx, const float* x, double* out, void* stream)
+{
+    if (ctx == nullptr || x == nullptr || out == nullptr) return SAPS_ERR_INVALID;
+    if (ctx->partials == nullptr) {
+        void* p = nullptr;
+        if (cudaMalloc(&p, (size_t)ctx->ntiles * sizeof(double)) != cudaSuccess) {
+            cudaGetLastError();
+            return SAPS_ERR_NOMEM;
+        }
+        ctx->partials = static_cast<double*>(p);
+    }
+    return launch_consensus(x, (size_t)ctx->ld, (uint32_t)ctx->N, ctx->n, ctx->ntiles, ctx->partials, out,
+                            (cudaStream_t)stream) == cudaSuccess
+               ? SAPS_OK
+               : SAPS_ERR_CUDA;
+}
+
+int saps_comm_stats(const saps_ctx* ctx, const double* bandwidth, const int32_t* pairs, uint64_t count,
+                    double bits_per_s_per_unit, double* out5)
+{
+    if (ctx == nullptr || bandwidth == nullptr || out5 == nullptr || !(bits_per_s_per_unit > 0.0)) return SAPS_ERR_INVALID;
+    const int n = ctx->n;
+    const int rc = check_pairs(n, pairs);
+    if (rc != SAPS_OK) return rc;
+    double lo = 0.0, sum = 0.0;
+    int links = 0;
+    for (int i = 0; i < n; ++i) {
+        const int j = pairs[i];
+        if (j <= i) continue;
+        const double a = bandwidth[(size_t)i * n + j], b = bandwidth[(size_t)j * n + i];
+        const double bw = a < b ? a : b;
+        if (links == 0 || bw < lo) lo = bw;
+        sum += bw;
+        ++links;
+    }
+    out5[0] = 2.0 * (double)count;                       // values sent + received per matched worker
+    out5[1] = 8.0 * (double)count;                       // the same in bytes (fp32)
+    out5[2] = links ? lo : 0.0;                          // bottleneck bandwidth of the round
+    out5[3] = links ? sum / links : 0.0;                 // mean bandwidth of the chosen links
+    out5[4] = (links && lo > 0.0) ? 32.0 * (double)count / (lo * bits_per_s_per_unit) : 0.0;  // seconds
+    return SAPS_OK;
+}
+
+int saps_debug_inject(saps_ctx* ctx, uint32_t skip_tile, uint32_t spin_limit)
+{
+    if (ctx == nullptr) return SAPS_ERR_INVALID;
+    ctx->skip_tile = skip_tile;
+    ctx->spin_limit = spin_limit == 0 ? kSpinLimit : spin_limit;
+    return SAPS_OK;
+}
+
 int saps_set_timing_events(saps_ctx* ctx, void* before, void* after)
 {
     if (ctx == nullptr) return SAPS_ERR_INVALID;
@@ -289,7 +382,8 @@ int saps_pack(saps_ctx* ctx, const float* x, uint64_t t, double keep_frac, float
     a.out_idx = out_idx;
     a.out_count = out_count;
     a.scratch = scratch_view(ctx->scratch, ctx->ntiles);
-    a.spin_limit = kSpinLimit;
+    a.spin_limit = ctx->spin_limit;
+    a.skip_tile = ctx->skip_tile;
     return launch_pack(a, (cudaStream_t)stream) == cudaSuccess ? SAPS_OK : SAPS_ERR_CUDA;
 }
 
@@ -311,7 +405,8 @@ int saps_pack_noalloc(saps_ctx* ctx, const float* x, uint64_t t, double keep_fra
     a.out_vals = out_vals;
     a.out_idx = out_idx;
     a.out_count = out_count;
-    a.spin_limit = kSpinLimit;
+    a.spin_limit = ctx->spin_limit;
+    a.skip_tile = ctx->skip_tile;
     if (launch_pack_static(a, ctx->ntiles, out_status, (cudaStream_t)stream) != cudaSuccess) {
         cudaGetLastError();
         return SAPS_ERR_CUDA;
@@ -345,7 +440,8 @@ int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, const int
     p.out_idx = out_idx;
     p.out_count = out_count;
     p.scratch = scratch_view(ctx->scratch, ctx->ntiles);
-    p.spin_limit = kSpinLimit;
+    p.spin_limit = ctx->spin_limit;
+    p.skip_tile = ctx->skip_tile;
     if (launch_pack(p, (cudaStream_t)stream) != cudaSuccess) return SAPS_ERR_CUDA;
     // pass 2: the fused round writes each worker's kept values at the scanned ranks
     const RowGroups rg = make_groups(ctx->n, pairs, true);
@@ -396,12 +492,17 @@ int saps_set_select_state(saps_ctx* ctx, const int64_t* R, uint64_t last_t)
 }
 
 int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t t_first, uint64_t T,
-                    double keep_frac, const int32_t* pairs_list, const double* bandwidth,
-                    int32_t* out_pairs_log, void* stream)
+                    double keep_frac, const float* lr_list, const int32_t* pairs_list,
+                    const double* bandwidth, int32_t* out_pairs_log, void* stream)
 {
     int rc = check_round_args(ctx, x, g, lr, t_first, keep_frac);
     if (rc != SAPS_OK) return rc;
     if (pairs_list == nullptr && bandwidth == nullptr) return SAPS_ERR_INVALID;
+    if (lr_list != nullptr) {
+        if (g == nullptr) return SAPS_ERR_INVALID;
+        for (uint64_t r = 0; r < T; ++r)
+            if (lr_list[r] != lr_list[r]) return SAPS_ERR_INVALID;
+    }
     const int n = ctx->n;
     int32_t chosen[kMaxWorkers];
     for (uint64_t r = 0; r < T; ++r) {
@@ -418,7 +519,8 @@ int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t 
         if (rc != SAPS_OK) return rc;
         if (out_pairs_log != nullptr) std::memcpy(out_pairs_log + r * (uint64_t)n, pairs, sizeof(int32_t) * n);
         const RowGroups rg = make_groups(n, pairs, g != nullptr);
-        const RoundArgs a = round_args(ctx, x, g, lr, rg, make_key(ctx->seed, t, keep_frac));
+        const float lr_t = lr_list != nullptr ? lr_list[r] : lr;
+        const RoundArgs a = round_args(ctx, x, g, lr_t, rg, make_key(ctx->seed, t, keep_frac));
         if (launch_round(a, false, (cudaStream_t)stream) != cudaSuccess) return SAPS_ERR_CUDA;
     }
     return SAPS_OK;
@@ -500,7 +602,8 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
         p.out_idx = pack->idx_host != nullptr ? pack->d_idx : nullptr;
         p.out_count = pack->d_count;
         p.scratch = sv;
-        p.spin_limit = kSpinLimit;
+        p.spin_limit = ctx->spin_limit;
+    p.skip_tile = ctx->skip_tile;
         failed |= launch_pack(p, ctx->lane_stream[0]) != cudaSuccess;
         failed |= cudaEventRecord(ctx->lane_event[0], ctx->lane_stream[0]) != cudaSuccess;
         for (int l = 1; l < saps_ctx::kLanes; ++l)

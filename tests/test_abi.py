@@ -82,7 +82,12 @@ def test_round_rejects_bad_arguments_before_any_launch():
     assert sb._lib.saps_pack(ctx, fake, 1, 0.5, None, fake, fake, None) == sb.SAPS_ERR_INVALID
     assert sb._lib.saps_pack(ctx, fake, 1, 2.0, fake, fake, fake, None) == sb.SAPS_ERR_INVALID
     assert sb._lib.saps_mask(ctx, 0, 0.5, fake, None) == sb.SAPS_ERR_INVALID
-    assert sb._lib.saps_run_rounds(ctx, fake, fake, 0.1, 1, 3, 0.5, None, None, None, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_run_rounds(ctx, fake, fake, 0.1, 1, 3, 0.5, None, None, None, None, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_set_update_order(ctx, 2) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_set_update_order(ctx, sb.SAPS_ORDER_GOSSIP_FIRST) == sb.SAPS_OK
+    assert sb._lib.saps_unpack_avg(ctx, fake, None, fake, fake, 0.5, None, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_unpack_avg(ctx, fake, fake, fake, fake, 0.5, sb._pairs([1, 2, 0, 3]), None) == sb.SAPS_ERR_PAIRS
+    assert sb._lib.saps_consensus_distance(ctx, fake, None, None) == sb.SAPS_ERR_INVALID
     assert sb._lib.saps_set_column_offset(ctx, (1 << 32) - 50) == sb.SAPS_ERR_INVALID
     assert sb._lib.saps_set_column_offset(ctx, (1 << 32) - 100) == sb.SAPS_OK
     sb.saps_destroy(ctx)
@@ -265,3 +270,36 @@ def test_select_peers_odd_n_missing_links_and_bad_input():
     pairs = sb.saps_select_peers(ctx, B2, 9, 4)
     assert pairs[0] != 1
     sb.saps_destroy(ctx)
+
+
+def test_comm_stats_table_1_and_bottleneck_bandwidth():
+    # Table 1: a worker moves 2 N/c values per round; Section IV-D: the round is as fast as
+    # the slowest chosen link
+    n = 4
+    B = np.array([[0, 10, 3, 4], [12, 0, 5, 6], [3, 5, 0, 2], [4, 6, 8, 0]], dtype=np.float64)
+    ctx = sb.saps_create(n, 100, 0)
+    st = sb.saps_comm_stats(ctx, B, [1, 0, 3, 2], 1000, 1e6)
+    assert st["values_per_worker"] == 2000 and st["bytes_per_worker"] == 8000
+    assert st["bottleneck_bandwidth"] == 2.0          # min(2, 8) on link (2,3); link (0,1) is min(10,12)
+    assert st["mean_bandwidth"] == 6.0
+    assert st["comm_time_s"] == 32 * 1000 / 2e6
+    st = sb.saps_comm_stats(ctx, B, [0, 1, 2, 3], 1000, 1e6)
+    assert st["bottleneck_bandwidth"] == 0.0 and st["comm_time_s"] == 0.0
+    with pytest.raises(sb.SapsError):
+        sb.saps_comm_stats(ctx, B, [1, 1, 3, 2], 10, 1e6)
+    sb.saps_destroy(ctx)
+
+
+def test_adaptive_selection_beats_random_matching_on_bottleneck_bandwidth():
+    # the point of Algorithm 3 (Fig. 5): the chosen pairs sit on faster links than random ones
+    n = 32
+    B = synth.bandwidth_matrix(n, 0.01, 5.0, seed=11)          # U(0, 5] MB/s as in Section IV-D
+    ctx = sb.saps_create(n, 100, 11)
+    rng = synth.matching_rng(11)
+    ours, rand = [], []
+    for t in range(1, 201):
+        pairs = sb.saps_select_peers(ctx, B, t, n)
+        ours.append(sb.saps_comm_stats(ctx, B, pairs, 1, 8e6)["mean_bandwidth"])
+        rand.append(sb.saps_comm_stats(ctx, B, synth.random_perfect_matching(n, rng), 1, 8e6)["mean_bandwidth"])
+    sb.saps_destroy(ctx)
+    assert np.mean(ours) > 1.25 * np.mean(rand)

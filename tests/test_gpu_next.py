@@ -1,0 +1,193 @@
+"""GPU parity of the widened path: Eq. 7 update order, per-round learning rates, the receiving
+side of the exchange (unpack-average), the consensus distance, and the bounded wait."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2002_09692_b200 import synth
+from gpu_util import DeviceMatrix, assert_bits_equal, round_up, torch_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sb():
+    torch_cuda()
+    from paper_2002_09692_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("N,ld", [(7, 7), (2050, 2052), (40_003, 40_032), (40_003, 40_003), (5 * 2048, 5 * 2048)])
+@pytest.mark.parametrize("p", [0.0, 0.1, 1.0])
+def test_eq7_order_round_and_emission(sb, N, ld, p):
+    torch = torch_cuda()
+    n, lr = 6, 0.1
+    pairs = [1, 0, 2, 5, 4, 3]
+    x = synth.gaussian_matrix(n, N, 1.0, 23, 0)
+    g = synth.gaussian_matrix(n, N, 0.05, 23, 1)
+    ctx = sb.saps_create_ld(n, N, ld, 23)
+    sb.saps_set_update_order(ctx, sb.SAPS_ORDER_GOSSIP_FIRST)
+    # plain round
+    dx, dg = DeviceMatrix(x, ld), DeviceMatrix(g, ld)
+    sb.saps_round(ctx, dx.ptr, dg.ptr, lr, pairs, 3, p)
+    want = x.copy()
+    m = oracle.gossip_round_eq7(want, g, lr, pairs, 23, 3, p)
+    torch.cuda.synchronize()
+    assert_bits_equal(dx.host(), want, "Eq. 7 order")
+    assert dx.canaries_intact()
+    # with emission: the wire buffer holds the current model x (nothing subtracted yet)
+    dx2 = DeviceMatrix(x, ld)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.full((n * cap,), 123.0, dtype=torch.float32, device="cuda")
+    idx = torch.full((cap,), -1, dtype=torch.int32, device="cuda")
+    count = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    sb.saps_round_pack(ctx, dx2.ptr, dg.ptr, lr, pairs, 3, p, vals, idx, count)
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    wv, wi, wc = oracle.pack(x, m, cap)
+    assert int(count[0]) == wc
+    assert_bits_equal(vals.cpu().numpy().reshape(n, cap)[:, :wc], wv[:, :wc], "Eq. 7 wire buffer")
+    assert_bits_equal(dx2.host(), want, "Eq. 7 order with emission")
+    # switching back restores Algorithm 2's order
+    sb.saps_set_update_order(ctx, sb.SAPS_ORDER_SGD_FIRST)
+    dx3 = DeviceMatrix(x, ld)
+    sb.saps_round(ctx, dx3.ptr, dg.ptr, lr, pairs, 3, p)
+    torch.cuda.synchronize()
+    want2 = x.copy()
+    oracle.gossip_round(want2, g, lr, pairs, 23, 3, p)
+    assert_bits_equal(dx3.host(), want2, "Algorithm 2 order")
+    sb.saps_destroy(ctx)
+
+
+def test_run_rounds_with_learning_rate_schedule(sb):
+    torch = torch_cuda()
+    n, N, T, p = 8, 20_000, 9, 0.2
+    x = synth.gaussian_matrix(n, N, 0.05, 24, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, 24, 1)
+    rng = synth.matching_rng(24)
+    plist = np.stack([synth.random_perfect_matching(n, rng) for _ in range(T)]).astype(np.int32)
+    lrs = (0.1 / np.sqrt(np.arange(1, T + 1))).astype(np.float32)       # gamma_t = gamma / sqrt(t)
+    for order, fn in ((0, oracle.gossip_round), (1, oracle.gossip_round_eq7)):
+        dx, dg = DeviceMatrix(x, round_up(N, 32)), DeviceMatrix(g, round_up(N, 32))
+        ctx = sb.saps_create_ld(n, N, round_up(N, 32), 24)
+        sb.saps_set_update_order(ctx, order)
+        sb.saps_run_rounds(ctx, dx.ptr, dg.ptr, 0.0, 1, T, p, pairs_list=plist, lr_list=lrs)
+        torch.cuda.synchronize()
+        sb.saps_destroy(ctx)
+        want = x.copy()
+        for t in range(1, T + 1):
+            fn(want, g, float(lrs[t - 1]), plist[t - 1], 24, t, p)
+        assert_bits_equal(dx.host(), want, f"schedule, order {order}")
+
+
+@pytest.mark.parametrize("N,p", [(33, 0.5), (70_001, 0.05), (300_000, 0.01), (4096, 1.0), (5000, 0.0)])
+def test_wire_path_sgd_pack_exchange_unpack(sb, N, p):
+    # SGD-only round -> saps_pack -> (buffers travel) -> saps_unpack_avg  ==  fused saps_round
+    torch = torch_cuda()
+    n, lr = 6, 0.05
+    pairs = [3, 4, 2, 0, 1, 5]                  # workers 2 and 5 have no peer
+    x = synth.gaussian_matrix(n, N, 1.0, 25, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, 25, 1)
+    ld = round_up(N, 4)
+    ctx = sb.saps_create_ld(n, N, ld, 25)
+    fused, dg = DeviceMatrix(x, ld), DeviceMatrix(g, ld)
+    sb.saps_round(ctx, fused.ptr, dg.ptr, lr, pairs, 2, p)
+    wire = DeviceMatrix(x, ld)
+    sb.saps_round(ctx, wire.ptr, dg.ptr, lr, list(range(n)), 2, p)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    count = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sb.saps_pack(ctx, wire.ptr, 2, p, vals, idx, count)
+    sb.saps_unpack_avg(ctx, wire.ptr, vals, idx, count, p, pairs)
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    assert_bits_equal(wire.host(), fused.host(), "wire path vs fused round")
+    assert wire.canaries_intact()
+    # against the oracle's receiving side, with an explicitly permuted receive buffer
+    a = x.copy()
+    oracle.sgd(a, g, lr)
+    m = oracle.mask(25, 2, p, N)
+    wv, wi, wc = oracle.pack(a, m, cap)
+    recv_host = np.ascontiguousarray(wv[pairs])
+    want = a.copy()
+    oracle.unpack_avg(want, recv_host, wi, min(wc, cap))
+    recv_dev = torch.from_numpy(recv_host).cuda()
+    wire2 = DeviceMatrix(a, ld)
+    sb.saps_unpack_avg(ctx, wire2.ptr, recv_dev, idx, count, p, None)      # row i = what i received
+    torch.cuda.synchronize()
+    assert_bits_equal(wire2.host(), want, "unpack-average, pairs=None")
+    sb.saps_destroy(ctx)
+
+
+@pytest.mark.parametrize("n,N,ld", [(2, 1, 1), (4, 2049, 2052), (32, 100_003, 100_032), (64, 5000, 5000)])
+def test_consensus_distance(sb, n, N, ld):
+    torch = torch_cuda()
+    x = synth.gaussian_matrix(n, N, 0.05, 26, 0)
+    x += np.float32(3.0)                        # a large common offset: deviations are small against it
+    dx = DeviceMatrix(x, ld)
+    ctx = sb.saps_create_ld(n, N, ld, 26)
+    out = torch.zeros(2, dtype=torch.float64, device="cuda")
+    sb.saps_consensus_distance(ctx, dx.ptr, out)
+    torch.cuda.synchronize()
+    want = oracle.consensus_distance(x)
+    got = float(out[0])
+    assert abs(got - want) <= 1e-10 * want + 1e-300, (got, want)
+    assert float(out[1]) == 0.0
+    # reproducible: the same bits on a second call
+    out2 = torch.zeros(1, dtype=torch.float64, device="cuda")
+    sb.saps_consensus_distance(ctx, dx.ptr, out2)
+    assert float(out2[0]) == got
+    # identical workers: exactly zero
+    same = np.repeat(x[:1], n, axis=0)
+    ds = DeviceMatrix(same, ld)
+    sb.saps_consensus_distance(ctx, ds.ptr, out)
+    torch.cuda.synchronize()
+    assert float(out[0]) == 0.0
+    sb.saps_destroy(ctx)
+
+
+def test_consensus_distance_follows_lemma_2_on_the_gpu(sb):
+    # sparse gossip contracts the consensus distance by q + p * lambda2 per round (Lemma 2)
+    torch = torch_cuda()
+    n, N, p = 32, 300_000, 0.25
+    x = synth.gaussian_matrix(n, N, 1.0, 27, 0)
+    dx = DeviceMatrix(x, round_up(N, 32))
+    ctx = sb.saps_create_ld(n, N, round_up(N, 32), 27)
+    rng = synth.matching_rng(27)
+    out = torch.zeros(7, dtype=torch.float64, device="cuda")
+    sb.saps_consensus_distance(ctx, dx.ptr, out[0:])
+    for t in range(1, 7):
+        sb.saps_round(ctx, dx.ptr, None, 0.0, synth.random_perfect_matching(n, rng), t, p)
+        sb.saps_consensus_distance(ctx, dx.ptr, out[t:])
+    torch.cuda.synchronize()
+    sb.saps_destroy(ctx)
+    d = out.cpu().numpy()
+    phat = oracle.threshold(p) / 2.0 ** 32
+    want = (1 - phat) + phat * (n - 2) / (2.0 * (n - 1))
+    ratios = d[1:] / d[:-1]
+    assert abs(ratios[0] - want) < 0.01 * want and abs(ratios.mean() - want) < 0.01 * want
+
+
+def test_bounded_wait_reports_a_timeout_instead_of_hanging(sb):
+    # one look-back tile never publishes; its successors give up after a short poll budget and the
+    # kernel returns with SAPS_ERR_TIMEOUT in the status word; the context stays usable
+    torch = torch_cuda()
+    n, N, p = 2, 40 * 2048, 0.05
+    x = synth.gaussian_matrix(n, N, 1.0, 28, 0)
+    dx = DeviceMatrix(x, N)
+    ctx = sb.saps_create(n, N, 28)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    count = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sb.saps_debug_inject(ctx, 3, 200)                       # tile 3 stays silent, 200 polls
+    sb.saps_pack(ctx, dx.ptr, 1, p, vals, idx, count)
+    assert sb.saps_status(ctx) == sb.SAPS_ERR_TIMEOUT
+    sb.saps_debug_inject(ctx, 0xFFFFFFFF, 0)                # hook off, default budget
+    sb.saps_pack(ctx, dx.ptr, 1, p, vals, idx, count)
+    assert sb.saps_status(ctx) == 0
+    wv, wi, wc = oracle.pack(x, oracle.mask(28, 1, p, N), cap)
+    assert int(count[0]) == wc
+    assert_bits_equal(vals.cpu().numpy()[:, :wc], wv[:, :wc], "pack after a timed-out call")
+    sb.saps_destroy(ctx)
