@@ -33,7 +33,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per worker-parameter of the fused round kernel, from the ncu
 # capture of that kernel on a smaller workload (summary under profiles/; traffic grows in proportion
 # to n*N).  Set to None whenever round_kernels.cu changes until the counters are retaken.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = 11.792
+NCU_TRAFFIC_BYTES_PER_ELEMENT = 11.784
 
 
 def parse_args():
@@ -290,6 +290,34 @@ def run_ours(args):
             "traffic": None if NCU_TRAFFIC_BYTES_PER_ELEMENT is None else NCU_TRAFFIC_BYTES_PER_ELEMENT * n * N,
         },
     }
+
+    # the other entry points of the path, timed alone on the same resident inputs (context only)
+    def timed(fn, reps=20):
+        for i in range(3):
+            fn(t + i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(reps):
+            fn(t + 3 + i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    pairs_fixed = sb.saps_select_peers(ctx, B, t, n)
+    t += 1
+    ms_round = timed(lambda tt: sb.saps_round(ctx, x, g, w.lr, pairs_fixed, tt, p, stream))
+    ms_pack = timed(lambda tt: sb.saps_pack(ctx, x, tt, p, vals, idx, count, stream))
+    dist_out = torch.zeros(1, dtype=torch.float64, device="cuda")
+    ms_dist = timed(lambda tt: sb.saps_consensus_distance(ctx, x, dist_out, stream))
+    result["other_entry_points"] = {
+        "saps_round": {"ms": ms_round, "algorithmic_gbs": bytes_round / (ms_round * 1e-3) / 1e9,
+                       "frac_of_measured_peak": bytes_round / (ms_round * 1e-3) / 1e9 / peak},
+        "saps_pack": {"ms": ms_pack, "algorithmic_bytes": 8.0 * n * kept + 4.0 * kept},
+        "saps_consensus_distance": {"ms": ms_dist, "algorithmic_gbs": 4.0 * n * N / (ms_dist * 1e-3) / 1e9,
+                                    "frac_of_measured_peak": 4.0 * n * N / (ms_dist * 1e-3) / 1e9 / peak},
+    }
+    t += 30
 
     if rank == 0 and not args.no_e2e:
         result["e2e"] = measure_e2e(args, sb, synth, w, ctx, B, t, x, g)

@@ -203,6 +203,7 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const PackArgs a)
     const uint64_t col0 = (uint64_t)tile * kTileCols;
 
     uint32_t cnt = 0;
+#pragma unroll 8
     for (int s = 0; s < kWords; ++s) {
         const uint64_t k = col0 + s * 32 + lane;
         const bool kept = (k < a.N) && column_kept(a.col_offset + (uint32_t)k, a.key);
@@ -276,22 +277,58 @@ __global__ void __launch_bounds__(kThreads) unpack_avg_kernel(const UnpackArgs a
 
 // Consensus distance, one block per column tile.  Per column the deviations are taken from
 // worker 0's value (exact in fp64), sum d^2 - (sum d)^2 / n, so that identical workers give
-// exactly zero and nearly identical ones lose no digits.
+// exactly zero and nearly identical ones lose no digits.  VEC = 4 streams 128-bit vectors.
+template <int VEC>
 __global__ void __launch_bounds__(kThreads) consensus_partial_kernel(const float* __restrict__ x, size_t ld,
                                                                      uint32_t N, int n, double* partials)
 {
+    constexpr int U = kTileCols / (kThreads * VEC);
     __shared__ double s_part[kThreads / 32];
     const int tid = threadIdx.x;
     double acc = 0.0;
     const uint64_t col0 = (uint64_t)blockIdx.x * kTileCols;
-#pragma unroll 2
-    for (int u = 0; u < kTileCols / kThreads; ++u) {
-        const uint64_t k = col0 + (uint64_t)u * kThreads + tid;
-        if (k < N) {
-            const double pivot = (double)__ldcs(x + k);
+    const uint32_t nfull = (VEC == 4) ? (N & ~3u) : N;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint64_t k = col0 + (uint64_t)(u * kThreads + tid) * VEC;
+        if (k < nfull) {
+            double pivot[VEC], sd[VEC], sdd[VEC];
+            if constexpr (VEC == 4) {
+                const float4 p = __ldcs(reinterpret_cast<const float4*>(x + k));
+                pivot[0] = p.x; pivot[1] = p.y; pivot[2] = p.z; pivot[3] = p.w;
+            } else {
+                pivot[0] = __ldcs(x + k);
+            }
+#pragma unroll
+            for (int c = 0; c < VEC; ++c) sd[c] = sdd[c] = 0.0;
+#pragma unroll 4
+            for (int i = 1; i < n; ++i) {
+                float v[VEC];
+                if constexpr (VEC == 4) {
+                    const float4 q = __ldcs(reinterpret_cast<const float4*>(x + (size_t)i * ld + k));
+                    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+                } else {
+                    v[0] = __ldcs(x + (size_t)i * ld + k);
+                }
+#pragma unroll
+                for (int c = 0; c < VEC; ++c) {
+                    const double d = (double)v[c] - pivot[c];
+                    sd[c] += d;
+                    sdd[c] += d * d;
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < VEC; ++c) acc += sdd[c] - sd[c] * sd[c] / (double)n;
+        }
+    }
+    if constexpr (VEC == 4) {
+        // the last (N mod 4) columns
+        const uint32_t k = nfull + tid;
+        if (k < N && col0 <= nfull && nfull < col0 + kTileCols) {
+            const double pivot = (double)x[k];
             double sd = 0.0, sdd = 0.0;
             for (int i = 1; i < n; ++i) {
-                const double d = (double)__ldcs(x + (size_t)i * ld + k) - pivot;
+                const double d = (double)x[(size_t)i * ld + k] - pivot;
                 sd += d;
                 sdd += d * d;
             }
@@ -337,7 +374,10 @@ cudaError_t launch_unpack_avg(const UnpackArgs& a, cudaStream_t stream)
 cudaError_t launch_consensus(const float* x, size_t ld, uint32_t N, int n, uint32_t ntiles, double* partials,
                              double* out, cudaStream_t stream)
 {
-    consensus_partial_kernel<<<ntiles, kThreads, 0, stream>>>(x, ld, N, n, partials);
+    if (ld % 4 == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0)
+        consensus_partial_kernel<4><<<ntiles, kThreads, 0, stream>>>(x, ld, N, n, partials);
+    else
+        consensus_partial_kernel<1><<<ntiles, kThreads, 0, stream>>>(x, ld, N, n, partials);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     consensus_final_kernel<<<1, kThreads, 0, stream>>>(partials, ntiles, out);
