@@ -14,7 +14,9 @@ back through the cycle.
 Readings taken where Algorithm 3 and Section II-C leave a choice
   * B is symmetrised by the elementwise minimum (Section II-C) and its diagonal
     is ignored.
-  * B*_ij = 1 iff B_ij >= B_thres (GetNewConnectedGraph of Algorithm 1).
+  * B*_ij = 1 iff B_ij >= B_thres (GetNewConnectedGraph of Algorithm 1) and the
+    link exists (B_ij > 0).  B_thres = inf stands for the bottleneck threshold:
+    the largest one that still lets as many workers pair up as the link graph allows.
   * An edge is "recently connected" iff R_ij > t - T_thres; an edge that never
     carried an exchange is never recent (R starts at NEVER).
   * IfStronglyConnected on the symmetric Q is plain undirected connectivity.
@@ -75,7 +77,7 @@ def new_timestamps(n: int) -> np.ndarray:
 def connected_graph(B, b_thres: float) -> np.ndarray:
     """GetNewConnectedGraph: B* as a boolean matrix."""
     S = symmetrise(B)
-    Bs = S >= b_thres
+    Bs = (S >= b_thres) & (S > 0.0)       # a zero entry means "no link at all"
     np.fill_diagonal(Bs, False)
     return Bs
 
@@ -226,9 +228,34 @@ def maximum_matching(E: np.ndarray, order=None) -> list[tuple[int, int]]:
 # Algorithm 3
 # ----------------------------------------------------------------------------
 
-def candidate_edges(B, R, t: int, b_thres: float, t_thres: int):
-    """Lines 1-5 of GenerateGossipMatrix: returns (E, mode)."""
+def bottleneck_threshold(B, order=None) -> float:
+    """The largest threshold for which B* = [B >= threshold] still admits a matching as large
+    as the whole link graph [B > 0] does: with it, the first-stage matching of Algorithm 3
+    maximises the slowest chosen link (the "bandwidth utilisation" of Section IV-D).  The
+    matching size can only shrink as the threshold rises, so a bisection over the sorted
+    link speeds finds it."""
     S = symmetrise(B)
+    n = S.shape[0]
+    speeds = sorted({float(S[i, j]) for i in range(n) for j in range(i + 1, n) if S[i, j] > 0.0})
+    if not speeds:
+        return 0.0
+    full = len(maximum_matching(S > 0.0, order))
+    lo, hi = 0, len(speeds) - 1          # speeds[lo] always works
+    while lo < hi:
+        mid = (lo + hi + 1) // 2
+        if len(maximum_matching(S >= speeds[mid], order)) == full:
+            lo = mid
+        else:
+            hi = mid - 1
+    return speeds[lo]
+
+
+def candidate_edges(B, R, t: int, b_thres: float, t_thres: int):
+    """Lines 1-5 of GenerateGossipMatrix: returns (E, mode).  b_thres = inf selects the
+    bottleneck threshold of this B."""
+    S = symmetrise(B)
+    if b_thres == float("inf"):
+        b_thres = bottleneck_threshold(B)
     Q = recent_graph(R, t, t_thres)
     if is_connected(Q):
         return connected_graph(B, b_thres), "bandwidth"

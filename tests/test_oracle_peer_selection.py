@@ -239,3 +239,27 @@ def test_recent_edges_stay_connected(n):
     assert later
     gaps = np.diff([warm] + later + [8 * t_thres])
     assert gaps.max() <= t_thres
+
+
+@pytest.mark.parametrize("n", [4, 6, 8])
+def test_bottleneck_threshold_against_brute_force(n):
+    # max over all perfect matchings of the slowest chosen link
+    for trial in range(15):
+        B = synth.bandwidth_matrix(n, 0.01, 5.0, seed=300 + 10 * n + trial)
+        S = ps.symmetrise(B)
+        best = max(min(S[a, b] for a, b in m) for m in all_perfect_matchings(n))
+        assert ps.bottleneck_threshold(B) == best
+        R = np.full((n, n), 50, dtype=np.int64)
+        pairs, info = ps.generate_gossip_matrix(B, R, 50, float("inf"), 5)
+        assert info["mode"] == "bandwidth" and len(info["match"]) == n // 2
+        assert min(S[i, pairs[i]] for i in range(n)) == best
+
+
+def test_bottleneck_threshold_with_missing_links_and_odd_n():
+    B = synth.bandwidth_matrix(5, 1.0, 9.0, seed=2)
+    S = ps.symmetrise(B)
+    theta = ps.bottleneck_threshold(B)
+    assert len(ps.maximum_matching(S >= theta)) == 2
+    bigger = [v for v in np.unique(S) if v > theta]
+    assert all(len(ps.maximum_matching(S >= v)) < 2 for v in bigger)
+    assert ps.bottleneck_threshold(np.zeros((4, 4))) == 0.0
