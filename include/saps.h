@@ -203,7 +203,10 @@ SAPS_API int saps_pack_noalloc(saps_ctx* ctx, const float* x, uint64_t t, double
 /* ---- peer selection (Algorithm 3; GetNewConnectedGraph of Algorithm 1) -------------------- */
 
 /* b_thres: links with min(B_ij, B_ji) >= b_thres form B*.  NaN selects the default, the
- * median of the symmetrised off-diagonal bandwidths of each call's matrix.
+ * median of the symmetrised off-diagonal bandwidths of each call's matrix.  +INFINITY selects,
+ * per call, the largest threshold for which B* still lets as many workers pair up as the
+ * link graph allows, so that the first matching maximises the slowest chosen link (the
+ * bandwidth utilisation measured in Section IV-D).
  * t_thres: an edge is "recently connected" iff R_ij > t - t_thres.  0 selects the default
  * max(2, 2 ceil(log2 n)). */
 SAPS_API int saps_set_select_params(saps_ctx* ctx, double b_thres, int t_thres);

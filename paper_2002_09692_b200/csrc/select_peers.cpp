@@ -153,6 +153,48 @@ int randomly_max_match(int n, const std::vector<uint8_t>& E, uint64_t seed, uint
     return pairs;
 }
 
+int matching_size(int n, const std::vector<uint8_t>& E)
+{
+    BlossomMatcher m(n, E);
+    const std::vector<int>& mate = m.solve();
+    int pairs = 0;
+    for (int v = 0; v < n; ++v) pairs += mate[v] > v;
+    return pairs;
+}
+
+// The largest threshold for which [B >= threshold] still admits a matching as large as the
+// whole link graph [B > 0]: the first-stage matching then maximises the slowest chosen link.
+// The matching size is monotone in the threshold, so bisect over the sorted link speeds.
+double bottleneck_threshold(int n, const std::vector<double>& B)
+{
+    std::vector<double> speeds;
+    for (int i = 0; i < n; ++i)
+        for (int j = i + 1; j < n; ++j)
+            if (B[(size_t)i * n + j] > 0.0) speeds.push_back(B[(size_t)i * n + j]);
+    if (speeds.empty()) return 0.0;
+    std::sort(speeds.begin(), speeds.end());
+    speeds.erase(std::unique(speeds.begin(), speeds.end()), speeds.end());
+    std::vector<uint8_t> E((size_t)n * n);
+    auto size_at = [&](double thr) {
+        for (int i = 0; i < n; ++i)
+            for (int j = 0; j < n; ++j) {
+                const double b = B[(size_t)i * n + j];
+                E[(size_t)i * n + j] = i != j && b > 0.0 && b >= thr;
+            }
+        return matching_size(n, E);
+    };
+    const int full = size_at(0.0);
+    size_t lo = 0, hi = speeds.size() - 1;
+    while (lo < hi) {
+        const size_t mid = (lo + hi + 1) / 2;
+        if (size_at(speeds[mid]) == full)
+            lo = mid;
+        else
+            hi = mid - 1;
+    }
+    return speeds[lo];
+}
+
 // FindConnectedSubgraph: component label per vertex; returns the number of components.
 int label_components(int n, const std::vector<uint8_t>& Q, std::vector<int>& label)
 {
@@ -193,7 +235,9 @@ int select_peers(SelectState& st, const double* bandwidth, uint64_t t, int32_t* 
             if (i != j) B[(size_t)i * n + j] = std::min(bandwidth[(size_t)i * n + j], bandwidth[(size_t)j * n + i]);
 
     double b_thres = st.b_thres;
-    if (st.b_thres_default) {
+    if (std::isinf(b_thres) && b_thres > 0.0) {
+        b_thres = bottleneck_threshold(n, B);
+    } else if (st.b_thres_default) {
         std::vector<double> links;
         for (int i = 0; i < n; ++i)
             for (int j = i + 1; j < n; ++j) links.push_back(B[(size_t)i * n + j]);

@@ -303,3 +303,45 @@ def test_adaptive_selection_beats_random_matching_on_bottleneck_bandwidth():
         rand.append(sb.saps_comm_stats(ctx, B, synth.random_perfect_matching(n, rng), 1, 8e6)["mean_bandwidth"])
     sb.saps_destroy(ctx)
     assert np.mean(ours) > 1.25 * np.mean(rand)
+
+
+@pytest.mark.parametrize("n", [4, 6, 8])
+def test_select_peers_bottleneck_mode_against_brute_force(n):
+    # b_thres = +inf: the chosen matching's slowest link is the best any perfect matching can do
+    for trial in range(12):
+        B = synth.bandwidth_matrix(n, 0.01, 5.0, seed=700 + 10 * n + trial)
+        S = ps.symmetrise(B)
+        best = max(min(S[a, b] for a, b in m) for m in all_perfect_matchings(n))
+        ctx = sb.saps_create(n, 16, trial)
+        sb.saps_set_select_params(ctx, float("inf"), 4)
+        sb.saps_set_select_state(ctx, [[90] * n for _ in range(n)], 90)      # bandwidth mode
+        pairs = sb.saps_select_peers(ctx, B, 90, n)
+        check_involution(pairs)
+        st = sb.saps_comm_stats(ctx, B, pairs, 1, 8e6)
+        assert st["bottleneck_bandwidth"] == best == ps.bottleneck_threshold(B)
+        sb.saps_destroy(ctx)
+
+
+def test_select_peers_bottleneck_mode_at_32_workers_matches_the_oracle():
+    n = 32
+    for trial in range(3):
+        B = synth.bandwidth_matrix(n, 0.01, 5.0, seed=40 + trial)
+        ctx = sb.saps_create(n, 16, trial)
+        sb.saps_set_select_params(ctx, float("inf"), 0)
+        sb.saps_set_select_state(ctx, [[7] * n for _ in range(n)], 7)
+        pairs = sb.saps_select_peers(ctx, B, 7, n)
+        check_involution(pairs)
+        assert all(pairs[i] != i for i in range(n))
+        st = sb.saps_comm_stats(ctx, B, pairs, 1, 8e6)
+        assert st["bottleneck_bandwidth"] == ps.bottleneck_threshold(B)
+        sb.saps_destroy(ctx)
+
+
+def test_bandwidth_study_orders_the_topologies():
+    # Section IV-D, Fig. 5: adaptive selection uses faster links than random matching or a ring
+    from paper_2002_09692_b200 import bandwidth_study
+    r = bandwidth_study.study(16, 8, 30, 1e-3, 5.0)
+    assert r["adaptive_bottleneck"]["slowest_link_mean"] > r["adaptive_median"]["slowest_link_mean"]
+    assert r["adaptive_median"]["slowest_link_mean"] > 2 * r["random_matching"]["slowest_link_mean"]
+    assert r["adaptive_median"]["mean_link_mean"] > r["random_matching"]["mean_link_mean"]
+    assert r["random_matching"]["slowest_link_mean"] > r["ring"]["slowest_link_mean"]
