@@ -33,7 +33,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per worker-parameter of the fused round kernel, from the ncu
 # capture of that kernel on a smaller workload (summary under profiles/; traffic grows in proportion
 # to n*N).  Set to None whenever round_kernels.cu changes until the counters are retaken.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = 11.784
+NCU_TRAFFIC_BYTES_PER_ELEMENT = 11.796
 
 
 def parse_args():
@@ -261,7 +261,7 @@ def run_ours(args):
     ms_per_step = elapsed_ms / K
     value = world * K / (elapsed_ms * 1e-3)
     bytes_round = 12.0 * n * N                       # read x, read g, write x
-    bytes_emit = 4.0 * n * kept                      # packed values written by the same pass
+    bytes_emit = 4.0 * n * kept + 4.0 * kept         # packed values and index list written by the same pass
     k_ms = statistics.mean(kernel_ms)
     achieved = (bytes_round + bytes_emit) / (k_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak_hbm()
@@ -273,7 +273,7 @@ def run_ours(args):
         "config": {
             "workload": f"{w.name}: n={n} workers, N={N} fp32 params each (per GPU), keep_frac={p}, "
                         f"lr={w.lr}, adaptive peer selection on U[{w.bw_range[0]:g},{w.bw_range[1]:g}] Mb/s",
-            "step": "saps_select_peers + saps_round_pack (mask scan kernel + fused SGD/mask/emit/average kernel)",
+            "step": "saps_select_peers + saps_round_pack (tile prefix-scan kernel + fused SGD/mask/emit/average kernel, which also counts the next round's mask per tile)",
             "row_stride": ld, "l2": f"inputs are {2 * 4 * n * N / 1e9:.2f} GB per step, far larger than the 126 MB L2",
             "sharding": "column shards, one per GPU, no collective" if world > 1 else "single GPU",
         },

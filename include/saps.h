@@ -121,6 +121,14 @@ SAPS_API int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, 
                     uint64_t t, double keep_frac, float* out_vals, uint32_t* out_idx,
                     uint32_t* out_count, void* stream);
 
+/* The emitting entry points need the number of kept columns per column tile before the fused
+ * kernel runs.  By default that kernel also counts them for round t+1 while it streams round
+ * t (the mask does not depend on the data, and the integer units are idle in a memory-bound
+ * kernel), so a following call for round t+1 with the same keep_frac only has to take a
+ * prefix sum of a few thousand numbers.  Any other call counts in a kernel of its own.
+ * Results are identical either way; enabled = 0 switches the run-ahead off. */
+SAPS_API int saps_set_run_ahead(saps_ctx* ctx, int enabled);
+
 /* Order of the two halves of the update.
  *   SAPS_ORDER_SGD_FIRST     Algorithm 2 (default): a = x - lr g, then the kept coordinates of
  *                            a matched pair become the mean of the two a's.

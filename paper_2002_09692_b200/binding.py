@@ -61,6 +61,7 @@ _SIGNATURES = {
     "saps_set_select_state": (_i32, [_vp, _vp, _u64]),
     "saps_run_rounds": (_i32, [_vp, _vp, _vp, _f32, _u64, _u64, _f64, _vp, _vp, _vp, _vp, _vp]),
     "saps_set_update_order": (_i32, [_vp, _i32]),
+    "saps_set_run_ahead": (_i32, [_vp, _i32]),
     "saps_unpack_avg": (_i32, [_vp, _vp, _vp, _vp, _vp, _f64, _vp, _vp]),
     "saps_consensus_distance": (_i32, [_vp, _vp, _vp, _vp]),
     "saps_comm_stats": (_i32, [_vp, _vp, _vp, _u64, _f64, _vp]),
@@ -241,6 +242,10 @@ SAPS_ORDER_GOSSIP_FIRST = 1
 
 def saps_set_update_order(ctx, order: int) -> None:
     _check(_lib.saps_set_update_order(ctx, order), "saps_set_update_order")
+
+
+def saps_set_run_ahead(ctx, enabled: bool) -> None:
+    _check(_lib.saps_set_run_ahead(ctx, int(bool(enabled))), "saps_set_run_ahead")
 
 
 def saps_unpack_avg(ctx, x, recv_vals, idx, count, keep_frac, pairs=None, stream=None) -> None:

@@ -78,7 +78,12 @@ struct RoundArgs {
     // emission of the wire buffer (all NULL/0 when not emitting)
     float* out_vals;
     uint32_t cap;
-    const uint32_t* tile_excl;
+    const uint32_t* tile_excl;   // exclusive prefix of kept columns per tile
+    uint32_t* out_idx;           // kept columns, written by the first row group (may be NULL)
+    // run-ahead for the next round: the first row group also counts, per tile, the columns
+    // that the NEXT round's mask keeps (NULL = off)
+    uint32_t* next_cnt;
+    RoundKey next_key;
 };
 
 cudaError_t launch_round(const RoundArgs& a, bool emit, cudaStream_t stream);
@@ -100,6 +105,13 @@ struct PackArgs {
 };
 
 cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream);
+
+// Mask scan without model data, in two small steps: kept columns per tile, then their
+// exclusive prefix, the total (out_count, may be NULL) and the overflow check.
+cudaError_t launch_mask_count(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t ntiles, uint32_t* tile_cnt,
+                              cudaStream_t stream);
+cudaError_t launch_tile_scan(const uint32_t* tile_cnt, uint32_t ntiles, uint32_t* tile_excl, uint32_t* out_count,
+                             uint32_t cap, int* status, cudaStream_t stream);
 
 cudaError_t launch_mask(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t* out_bits,
                         cudaStream_t stream);

@@ -178,76 +178,67 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
     }
 }
 
-// Mask scan without model data (indices, count, per-tile prefixes for the fused emission).
-// One block covers kScanSub column tiles, one warp each, so that the look-back chain has
-// eight times fewer links than tiles.
-constexpr int kScanSub = kThreads / 32;
-
-__global__ void __launch_bounds__(kThreads) scan_kernel(const PackArgs a)
+// Kept columns of every tile under one round's mask (no model data): one warp per tile.
+__global__ void __launch_bounds__(kThreads) mask_count_kernel(uint32_t N, uint32_t col_offset, RoundKey key,
+                                                             uint32_t ntiles, uint32_t* tile_cnt)
 {
-    constexpr int kWords = kTileCols / 32;  // mask words per tile
-    __shared__ uint32_t s_big, s_excl, s_abort;
-    __shared__ uint32_t s_cnt[kScanSub];
-    __shared__ uint32_t s_word[kScanSub][kWords];
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) {
-        s_big = atomicAdd(a.scratch.ticket, 1u);
-        s_abort = 0;
-    }
-    __syncthreads();
-    const uint32_t big = s_big;
-    const uint32_t nbig = (a.scratch.ntiles + kScanSub - 1) / kScanSub;
-    if (big >= nbig) return;
-    const uint32_t tile = big * kScanSub + warp;            // this warp's tile (may lie past the end)
+    const int lane = threadIdx.x & 31;
+    const uint32_t tile = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (tile >= ntiles) return;
     const uint64_t col0 = (uint64_t)tile * kTileCols;
-
     uint32_t cnt = 0;
 #pragma unroll 8
-    for (int s = 0; s < kWords; ++s) {
+    for (int s = 0; s < kTileCols / 32; ++s) {
         const uint64_t k = col0 + s * 32 + lane;
-        const bool kept = (k < a.N) && column_kept(a.col_offset + (uint32_t)k, a.key);
-        const uint32_t w = __ballot_sync(0xFFFFFFFFu, kept);
-        if (lane == 0) s_word[warp][s] = w;
-        cnt += __popc(w);
+        cnt += ((k < N) && column_kept(col_offset + (uint32_t)k, key)) ? 1u : 0u;
     }
-    if (lane == 0) s_cnt[warp] = cnt;
+    cnt = warp_sum(cnt);
+    if (lane == 0) tile_cnt[tile] = cnt;
+}
+
+// Exclusive prefix of the tile counts, the total and the overflow check: one block walks the
+// list in chunks of its size (a few chunks for tens of millions of columns).
+constexpr int kScanThreads = 1024;
+__global__ void __launch_bounds__(kScanThreads) tile_scan_kernel(const uint32_t* __restrict__ tile_cnt,
+                                                                 uint32_t ntiles, uint32_t* __restrict__ tile_excl,
+                                                                 uint32_t* out_count, uint32_t cap, int* status)
+{
+    __shared__ uint32_t s_warp[kScanThreads / 32];
+    __shared__ uint32_t s_carry;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) s_carry = 0;
     __syncthreads();
-    uint32_t before = 0, total = 0;
+    for (uint32_t base = 0; base < ntiles; base += kScanThreads) {
+        const uint32_t i = base + tid;
+        const uint32_t c = i < ntiles ? tile_cnt[i] : 0u;
+        uint32_t inc = c;
 #pragma unroll
-    for (int w = 0; w < kScanSub; ++w) {
-        const uint32_t c = s_cnt[w];
-        before += (w < warp) ? c : 0u;
-        total += c;
-    }
-    if (warp == 0) {
-        uint32_t excl;
-        const bool ok = lookback_exclusive(a.scratch, big, total, a.spin_limit, a.skip_tile, lane, &excl);
-        if (lane == 0) {
-            s_excl = excl;
-            if (!ok) s_abort = 1;
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+            if (lane >= d) inc += o;
         }
-    }
-    __syncthreads();
-    if (s_abort) return;
-    const uint32_t base = s_excl + before;
-    if (tile < a.scratch.ntiles) {
-        if (lane == 0) a.scratch.tile_excl[tile] = base;
-        if (a.out_idx != nullptr) {
-            uint32_t r = base;
-            for (int s = 0; s < kWords; ++s) {
-                const uint32_t w = s_word[warp][s];
-                if ((w >> lane) & 1u) {
-                    const uint32_t mine = r + __popc(w & ((1u << lane) - 1u));
-                    if (mine < a.cap) a.out_idx[mine] = a.col_offset + (uint32_t)(col0 + s * 32 + lane);
-                }
-                r += __popc(w);
+        if (lane == 31) s_warp[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            uint32_t w = s_warp[lane];
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, w, d);
+                if (lane >= d) w += o;
             }
+            s_warp[lane] = w;  // inclusive over warps
         }
+        __syncthreads();
+        const uint32_t carry = s_carry;
+        const uint32_t before = carry + (warp ? s_warp[warp - 1] : 0u) + inc - c;
+        if (i < ntiles) tile_excl[i] = before;
+        __syncthreads();
+        if (tid == kScanThreads - 1) s_carry = carry + s_warp[kScanThreads / 32 - 1];
+        __syncthreads();
     }
-    if (big == nbig - 1 && tid == 0) {
-        if (a.out_count != nullptr) *a.out_count = s_excl + total;
-        if (s_excl + total > a.cap) atomicCAS(a.scratch.status, 0, -4 /* SAPS_ERR_OVERFLOW */);
+    if (tid == 0) {
+        if (out_count != nullptr) *out_count = s_carry;
+        if (s_carry > cap) atomicCAS(status, 0, -4 /* SAPS_ERR_OVERFLOW */);
     }
 }
 
@@ -389,10 +380,7 @@ cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream)
     const uint32_t ntiles = a.scratch.ntiles;
     cudaError_t e = cudaMemsetAsync(a.scratch.ticket, 0, scratch_clear_bytes(ntiles), stream);
     if (e != cudaSuccess) return e;
-    if (a.out_vals != nullptr)
-        pack_kernel<true><<<ntiles, kThreads, 0, stream>>>(a);
-    else
-        scan_kernel<<<(ntiles + kScanSub - 1) / kScanSub, kThreads, 0, stream>>>(a);
+    pack_kernel<true><<<ntiles, kThreads, 0, stream>>>(a);
     return cudaGetLastError();
 }
 
@@ -435,6 +423,22 @@ cudaError_t launch_pack_static(PackArgs a, uint32_t ntiles, int* out_status, cud
     if (out_status != nullptr)
         e = cudaMemcpyAsync(out_status, a.scratch.status, sizeof(int), cudaMemcpyDeviceToDevice, stream);
     return e;
+}
+
+cudaError_t launch_mask_count(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t ntiles, uint32_t* tile_cnt,
+                              cudaStream_t stream)
+{
+    const uint32_t per_block = kThreads / 32;
+    mask_count_kernel<<<(ntiles + per_block - 1) / per_block, kThreads, 0, stream>>>(N, col_offset, key, ntiles,
+                                                                                    tile_cnt);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tile_scan(const uint32_t* tile_cnt, uint32_t ntiles, uint32_t* tile_excl, uint32_t* out_count,
+                             uint32_t cap, int* status, cudaStream_t stream)
+{
+    tile_scan_kernel<<<1, kScanThreads, 0, stream>>>(tile_cnt, ntiles, tile_excl, out_count, cap, status);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_mask(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t* out_bits,

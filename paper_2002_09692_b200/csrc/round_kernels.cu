@@ -151,6 +151,47 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
             running += all;
         }
         total = running - excl;
+        // the list of kept columns is the same for every row group: the first one writes it
+        if (blockIdx.y == 0 && a.out_idx != nullptr) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                uint32_t r = rank[u];
+#pragma unroll
+                for (int c = 0; c < VEC; ++c) {
+                    if ((bits[u] >> c) & 1u) {
+                        if (r < a.cap) a.out_idx[r] = a.col_offset + col[u] + c;
+                        ++r;
+                    }
+                }
+            }
+        }
+        // run-ahead: how many columns of this tile the next round's mask keeps
+        if (blockIdx.y == 0 && a.next_cnt != nullptr) {
+            __shared__ uint32_t s_next[kWarps];
+            uint32_t c = 0;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (inb[u]) {
+#pragma unroll
+                    for (int q = 0; q < VEC; ++q) c += column_kept(a.col_offset + col[u] + q, a.next_key) ? 1u : 0u;
+                }
+            }
+            if constexpr (VEC == 4) {
+                const uint32_t k = nfull + tid;  // the (N mod 4) leftover columns belong to the last tile
+                if (k < a.N && col_tile <= nfull && nfull < col_tile + kTileCols)
+                    c += column_kept(a.col_offset + k, a.next_key) ? 1u : 0u;
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, d);
+            if (lane == 0) s_next[warp] = c;
+            __syncthreads();
+            if (tid == 0) {
+                uint32_t t = 0;
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) t += s_next[w];
+                a.next_cnt[tile] = t;
+            }
+        }
         // what each worker sends: its value before the average (post-SGD in Algorithm 2's order)
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -222,6 +263,7 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
                     uint32_t r = excl + total;
                     for (uint32_t q = nfull; q < k; ++q) r += column_kept(a.col_offset + q, a.key) ? 1u : 0u;
                     if (r < a.cap) {
+                        if (blockIdx.y == 0 && a.out_idx != nullptr) a.out_idx[r] = a.col_offset + k;
                         a.out_vals[(size_t)ra * a.cap + r] = pa;
                         if (paired) a.out_vals[(size_t)rb * a.cap + r] = pb;
                     }

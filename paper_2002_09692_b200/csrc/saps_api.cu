@@ -31,6 +31,14 @@ struct saps_ctx {
     cudaStream_t lane_stream[kLanes];
     cudaEvent_t lane_event[kLanes];
     bool lanes_ready;
+    // Mask scan of the emitting round (saps_round_pack): kept columns per tile for the current
+    // round and, counted ahead by the fused kernel itself, for the next one; their prefix.
+    uint32_t* emit_mem;        // device: cnt[0][ntiles], cnt[1][ntiles], excl[ntiles]
+    int emit_cur;              // which cnt buffer the next call looks at
+    bool ahead_valid;          // cnt[emit_cur] holds the counts of round ahead_t ...
+    uint64_t ahead_t, ahead_thr;
+    uint32_t ahead_col_offset; // ... for this threshold and column offset
+    int run_ahead;             // 1 = let the fused kernel count the next round's mask (default)
     SelectState select;
 };
 
@@ -138,6 +146,9 @@ RoundArgs round_args(const saps_ctx* ctx, float* x, const float* g, float lr, co
     a.out_vals = nullptr;
     a.cap = 0;
     a.tile_excl = nullptr;
+    a.out_idx = nullptr;
+    a.next_cnt = nullptr;
+    a.next_key = key;
     return a;
 }
 
@@ -187,6 +198,12 @@ int saps_create_ld(int n, uint64_t N, uint64_t ld, uint64_t seed, saps_ctx** out
     ctx->scratch = nullptr;
     ctx->scratch_device = -1;
     ctx->lanes_ready = false;
+    ctx->emit_mem = nullptr;
+    ctx->emit_cur = 0;
+    ctx->ahead_valid = false;
+    ctx->ahead_t = ctx->ahead_thr = 0;
+    ctx->ahead_col_offset = 0;
+    ctx->run_ahead = 1;
     ctx->select.n = n;
     ctx->select.seed = seed;
     try {
@@ -214,6 +231,7 @@ int saps_destroy(saps_ctx* ctx)
         }
     if (ctx->scratch != nullptr) cudaFree(ctx->scratch);
     if (ctx->partials != nullptr) cudaFree(ctx->partials);
+    if (ctx->emit_mem != nullptr) cudaFree(ctx->emit_mem);
     delete ctx;
     return SAPS_OK;
 }
@@ -414,6 +432,63 @@ int saps_pack_noalloc(saps_ctx* ctx, const float* x, uint64_t t, double keep_fra
     return SAPS_OK;
 }
 
+namespace {
+
+int ensure_emit_memory(saps_ctx* ctx)
+{
+    if (ctx->emit_mem != nullptr) return SAPS_OK;
+    void* p = nullptr;
+    if (cudaMalloc(&p, (size_t)3 * ctx->ntiles * sizeof(uint32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        return SAPS_ERR_NOMEM;
+    }
+    ctx->emit_mem = static_cast<uint32_t*>(p);
+    return SAPS_OK;
+}
+
+// Everything the fused kernel needs to emit round t's wire buffer, enqueued on `stream`:
+// the per-tile counts of round t (taken from the previous call's run-ahead when they are
+// there, counted now otherwise), their prefix, the total.  Fills the emission fields of `a`
+// and arranges for the kernel to count round t+1 ahead.
+int prepare_emission(saps_ctx* ctx, uint64_t t, double keep_frac, uint32_t cap, uint32_t* out_idx,
+                     uint32_t* out_count, float* out_vals, cudaStream_t stream, RoundArgs* a)
+{
+    int rc = ensure_scratch(ctx);
+    if (rc != SAPS_OK) return rc;
+    rc = ensure_emit_memory(ctx);
+    if (rc != SAPS_OK) return rc;
+    const uint32_t nt = ctx->ntiles;
+    const uint64_t thr = threshold64(keep_frac);
+    uint32_t* cnt_now = ctx->emit_mem + (size_t)ctx->emit_cur * nt;
+    uint32_t* cnt_next = ctx->emit_mem + (size_t)(ctx->emit_cur ^ 1) * nt;
+    uint32_t* excl = ctx->emit_mem + (size_t)2 * nt;
+    const bool have = ctx->ahead_valid && ctx->ahead_t == t && ctx->ahead_thr == thr &&
+                      ctx->ahead_col_offset == (uint32_t)ctx->col_offset;
+    ctx->ahead_valid = false;
+    if (!have && launch_mask_count((uint32_t)ctx->N, (uint32_t)ctx->col_offset, make_key(ctx->seed, t, keep_frac), nt,
+                                   cnt_now, stream) != cudaSuccess)
+        return SAPS_ERR_CUDA;
+    if (launch_tile_scan(cnt_now, nt, excl, out_count, cap, static_cast<int*>(ctx->scratch), stream) != cudaSuccess)
+        return SAPS_ERR_CUDA;
+    a->out_vals = out_vals;
+    a->cap = cap;
+    a->tile_excl = excl;
+    a->out_idx = out_idx;
+    a->next_cnt = nullptr;
+    if (ctx->run_ahead && t + 1 != 0) {
+        a->next_cnt = cnt_next;
+        a->next_key = make_key(ctx->seed, t + 1, keep_frac);
+        ctx->ahead_valid = true;   // true once the kernel the caller enqueues next has run
+        ctx->ahead_t = t + 1;
+        ctx->ahead_thr = thr;
+        ctx->ahead_col_offset = (uint32_t)ctx->col_offset;
+        ctx->emit_cur ^= 1;
+    }
+    return SAPS_OK;
+}
+
+}  // namespace
+
 int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, const int32_t* pairs,
                     uint64_t t, double keep_frac, float* out_vals, uint32_t* out_idx,
                     uint32_t* out_count, void* stream)
@@ -423,33 +498,25 @@ int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, const int
     if (out_vals == nullptr || out_count == nullptr) return SAPS_ERR_INVALID;
     rc = check_pairs(ctx->n, pairs);
     if (rc != SAPS_OK) return rc;
-    rc = ensure_scratch(ctx);
-    if (rc != SAPS_OK) return rc;
     const RoundKey key = make_key(ctx->seed, t, keep_frac);
     const uint32_t cap = (uint32_t)saps_pack_capacity(ctx, keep_frac);
-    // pass 1 touches no model data: mask scan -> indices, count and per-tile prefixes
-    PackArgs p;
-    p.x = nullptr;
-    p.ld = (size_t)ctx->ld;
-    p.N = (uint32_t)ctx->N;
-    p.n = ctx->n;
-    p.key = key;
-    p.col_offset = (uint32_t)ctx->col_offset;
-    p.cap = cap;
-    p.out_vals = nullptr;
-    p.out_idx = out_idx;
-    p.out_count = out_count;
-    p.scratch = scratch_view(ctx->scratch, ctx->ntiles);
-    p.spin_limit = ctx->spin_limit;
-    p.skip_tile = ctx->skip_tile;
-    if (launch_pack(p, (cudaStream_t)stream) != cudaSuccess) return SAPS_ERR_CUDA;
-    // pass 2: the fused round writes each worker's kept values at the scanned ranks
+    // pass 1 touches no model data: kept columns per tile -> prefixes and count
     const RowGroups rg = make_groups(ctx->n, pairs, true);
     RoundArgs a = round_args(ctx, x, g, lr, rg, key);
-    a.out_vals = out_vals;
-    a.cap = cap;
-    a.tile_excl = p.scratch.tile_excl;
-    return timed_round(ctx, a, true, (cudaStream_t)stream);
+    rc = prepare_emission(ctx, t, keep_frac, cap, out_idx, out_count, out_vals, (cudaStream_t)stream, &a);
+    if (rc != SAPS_OK) return rc;
+    // pass 2: the fused round writes the kept columns and each worker's kept values at their ranks
+    rc = timed_round(ctx, a, true, (cudaStream_t)stream);
+    if (rc != SAPS_OK) ctx->ahead_valid = false;
+    return rc;
+}
+
+int saps_set_run_ahead(saps_ctx* ctx, int enabled)
+{
+    if (ctx == nullptr) return SAPS_ERR_INVALID;
+    ctx->run_ahead = enabled != 0;
+    ctx->ahead_valid = false;
+    return SAPS_OK;
 }
 
 int saps_set_select_params(saps_ctx* ctx, double b_thres, int t_thres)
@@ -575,10 +642,6 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
     if (rc != SAPS_OK) return rc;
     rc = ensure_lanes(ctx);
     if (rc != SAPS_OK) return rc;
-    if (pack != nullptr) {
-        rc = ensure_scratch(ctx);
-        if (rc != SAPS_OK) return rc;
-    }
     const int n = ctx->n;
     const uint64_t N = ctx->N;
     const uint64_t ld_dev = (N + 31) / 32 * 32;
@@ -587,24 +650,12 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
     const RoundKey key = make_key(ctx->seed, t, keep_frac);
     const uint32_t cap = emit ? (uint32_t)saps_pack_capacity(ctx, keep_frac) : 0;
     bool failed = false;
-    ScratchView sv{};
+    RoundArgs emit_args = round_args(ctx, d_x, g_host != nullptr ? d_g : nullptr, lr, rg, key, ld_dev);
     if (emit) {
-        sv = scratch_view(ctx->scratch, ctx->ntiles);
-        PackArgs p;
-        p.x = nullptr;
-        p.ld = (size_t)ld_dev;
-        p.N = (uint32_t)N;
-        p.n = n;
-        p.key = key;
-        p.col_offset = (uint32_t)ctx->col_offset;
-        p.cap = cap;
-        p.out_vals = nullptr;
-        p.out_idx = pack->idx_host != nullptr ? pack->d_idx : nullptr;
-        p.out_count = pack->d_count;
-        p.scratch = sv;
-        p.spin_limit = ctx->spin_limit;
-    p.skip_tile = ctx->skip_tile;
-        failed |= launch_pack(p, ctx->lane_stream[0]) != cudaSuccess;
+        // the mask scan touches no model data: it runs first on lane 0, the other lanes wait for it
+        rc = prepare_emission(ctx, t, keep_frac, cap, pack->idx_host != nullptr ? pack->d_idx : nullptr,
+                              pack->d_count, pack->d_vals, ctx->lane_stream[0], &emit_args);
+        if (rc != SAPS_OK) return rc;
         failed |= cudaEventRecord(ctx->lane_event[0], ctx->lane_stream[0]) != cudaSuccess;
         for (int l = 1; l < saps_ctx::kLanes; ++l)
             failed |= cudaStreamWaitEvent(ctx->lane_stream[l], ctx->lane_event[0], 0) != cudaSuccess;
@@ -622,14 +673,9 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
         if (g_host != nullptr)
             failed |= cudaMemcpy2DAsync(d_g + c0, ld_dev * sizeof(float), g_host + c0, N * sizeof(float), width,
                                         n, cudaMemcpyHostToDevice, s) != cudaSuccess;
-        RoundArgs a = round_args(ctx, d_x, g_host != nullptr ? d_g : nullptr, lr, rg, key, ld_dev);
+        RoundArgs a = emit_args;
         a.tile_begin = tb;
         a.tile_count = tc;
-        if (emit) {
-            a.out_vals = pack->d_vals;
-            a.cap = cap;
-            a.tile_excl = sv.tile_excl;
-        }
         failed |= launch_round(a, emit, s) != cudaSuccess;
         failed |= cudaMemcpy2DAsync(x_host + c0, N * sizeof(float), d_x + c0, ld_dev * sizeof(float), width, n,
                                     cudaMemcpyDeviceToHost, s) != cudaSuccess;
@@ -651,6 +697,7 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
     }
     for (int l = 0; l < saps_ctx::kLanes; ++l) failed |= cudaStreamSynchronize(ctx->lane_stream[l]) != cudaSuccess;
     if (failed) {
+        ctx->ahead_valid = false;
         cudaGetLastError();
         return SAPS_ERR_CUDA;
     }

@@ -205,3 +205,41 @@ def test_unfused_wire_path_equals_fused_round(sb):
     for i in range(n):
         assert_bits_equal(v[i], v[pairs[i]], "peers send identical buffers")
     sb.saps_destroy(ctx)
+
+
+@pytest.mark.parametrize("prefetch", [True, False])
+def test_round_pack_sequence_with_scan_run_ahead(sb, prefetch):
+    # consecutive rounds find their mask scan already done by the previous call; jumps in t,
+    # a changed keep_frac and a changed capacity fall back to an in-line scan; same results
+    torch = torch_cuda()
+    n, N = 4, 9 * 2048 + 77
+    ld = round_up(N, 32)
+    pairs = [1, 0, 3, 2]
+    x = synth.gaussian_matrix(n, N, 1.0, 91, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, 91, 1)
+    dx, dg = DeviceMatrix(x, ld), DeviceMatrix(g, ld)
+    ctx = sb.saps_create_ld(n, N, ld, 91)
+    sb.saps_set_run_ahead(ctx, prefetch)
+    want = x.copy()
+    schedule = [(1, 0.1), (2, 0.1), (3, 0.1), (10, 0.1), (11, 0.3), (12, 0.3), (12, 0.3), (13, 0.05)]
+    for step, (t, p) in enumerate(schedule):
+        if step == 5:
+            sb.saps_set_pack_capacity(ctx, 7000)
+        cap = sb.saps_pack_capacity(ctx, p)
+        vals = torch.full((n, cap), 123.0, dtype=torch.float32, device="cuda")
+        idx = torch.full((cap,), -1, dtype=torch.int32, device="cuda")
+        count = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+        sb.saps_round_pack(ctx, dx.ptr, dg.ptr, 0.05, pairs, t, p, vals, idx, count)
+        a = want.copy()
+        oracle.sgd(a, g, 0.05)
+        m = oracle.mask(91, t, p, N)
+        wv, wi, wc = oracle.pack(a, m, cap)
+        oracle.pair_average(a, pairs, m)
+        want = a
+        torch.cuda.synchronize()
+        assert int(count[0]) == wc, (step, t, p)
+        assert (idx.cpu().numpy().view(np.uint32)[:wc] == wi[:wc]).all(), (step, t, p)
+        assert_bits_equal(vals.cpu().numpy()[:, :wc], wv[:, :wc], f"wire buffer step {step}")
+        assert_bits_equal(dx.host(), want, f"model step {step}")
+    assert sb.saps_status(ctx) == 0
+    sb.saps_destroy(ctx)
