@@ -34,7 +34,7 @@
 #include <stdint.h>
 #include <math.h>
 
-/* ---- mask hash (this build's definition; all arithmetic wraps mod 2^32) -- */
+/* ---- mask hash (defined here, not by the paper; arithmetic wraps mod 2^32) -- */
 
 #define ORC_M1 0x9E3779B9u
 #define ORC_M2 0x6A09E667u
