@@ -319,8 +319,10 @@ def run_ours(args):
     }
     t += 30
 
-    if rank == 0 and not args.no_e2e:
-        result["e2e"] = measure_e2e(args, sb, synth, w, ctx, B, t, x, g)
+    if not args.no_e2e:
+        e2e = measure_e2e(args, sb, sharding, w, ctx, B, t, x, g, world, col_offset, barrier)
+        if rank == 0:
+            result["e2e"] = e2e
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = measure_cpu_baseline(args, synth, w)
 
@@ -332,16 +334,17 @@ def run_ours(args):
         print(json.dumps(result))
 
 
-def measure_e2e(args, sb, synth, w, ctx, B, t, x_dev, g_dev):
+def measure_e2e(args, sb, sharding, w, ctx, B, t, x_dev, g_dev, world, col_offset, barrier):
     """The same round through the host-buffer entry point: pinned host matrices in, updated
-    model out, copies inside the timed region."""
+    model out, copies inside the timed region.  Every rank runs it on its own column shard;
+    the time is the slowest rank's."""
     import torch
     n, N = w.n, w.N
     hx = torch.empty(n, N, dtype=torch.float32).pin_memory()
     hg = torch.empty(n, N, dtype=torch.float32).pin_memory()
     hx.copy_(x_dev[:, :N])
     hg.copy_(g_dev[:, :N])
-    sb.saps_set_column_offset(ctx, 0)
+    sb.saps_set_column_offset(ctx, col_offset)
     cap = sb.saps_pack_capacity(ctx, args.keep_frac)
     hv = torch.empty(n, cap, dtype=torch.float32).pin_memory()
     hi = torch.empty(cap, dtype=torch.int32).pin_memory()
@@ -358,13 +361,15 @@ def measure_e2e(args, sb, synth, w, ctx, B, t, x_dev, g_dev):
     for _ in range(2):
         step(t)
         t += 1
-    torch.cuda.synchronize()
+    barrier()
     t0 = time.perf_counter()
     for _ in range(steps):
         step(t)
         t += 1
     dt = time.perf_counter() - t0                     # the call waits for the copies back
-    return {"value": steps / dt, "unit": UNIT, "h2d_bytes_per_step": 2 * 4 * n * N,
+    dt = sharding.max_over_ranks(dt)
+    barrier()
+    return {"value": world * steps / dt, "unit": UNIT, "h2d_bytes_per_step": 2 * 4 * n * N,
             "d2h_bytes_per_step": 4 * n * N + 4 * n * cap + 4 * cap + 4, "ms_per_step": dt / steps * 1e3,
             "steps": steps, "kept_columns": int(hc.numpy().view("uint32")[0]),
             "api": "saps_select_peers + saps_round_pack_host (pinned host x and g in; x, packed values, "
