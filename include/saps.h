@@ -73,8 +73,9 @@ typedef struct saps_ctx saps_ctx;
  * object; no device work happens here). */
 SAPS_API int saps_create(int n, uint64_t N, uint64_t seed, saps_ctx** out);
 
-/* Same, with an explicit row stride ld >= N.  The 128-bit fast path of the round needs
- * ld % 4 == 0 and 16-byte aligned x and g; any other layout runs a scalar kernel. */
+/* Same, with an explicit row stride ld >= N.  The round uses the widest access every row
+ * start allows: 128-bit when ld % 4 == 0 and x, g are 16-byte aligned; 64-bit when ld % 2 == 0
+ * and they are 8-byte aligned; scalar otherwise.  All three give the same bits. */
 SAPS_API int saps_create_ld(int n, uint64_t N, uint64_t ld, uint64_t seed, saps_ctx** out);
 
 /* Column sharding (one shard per GPU): this context's column 0 is column col_offset of the

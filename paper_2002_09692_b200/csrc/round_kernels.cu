@@ -35,6 +35,9 @@ __device__ __forceinline__ Chunk<VEC> load_stream(const float* p)
     if constexpr (VEC == 4) {
         float4 t = __ldcs(reinterpret_cast<const float4*>(p));
         c.v[0] = t.x; c.v[1] = t.y; c.v[2] = t.z; c.v[3] = t.w;
+    } else if constexpr (VEC == 2) {
+        float2 t = __ldcs(reinterpret_cast<const float2*>(p));
+        c.v[0] = t.x; c.v[1] = t.y;
     } else {
         c.v[0] = __ldcs(p);
     }
@@ -46,6 +49,8 @@ __device__ __forceinline__ void store_stream(float* p, const Chunk<VEC>& c)
 {
     if constexpr (VEC == 4) {
         __stcs(reinterpret_cast<float4*>(p), make_float4(c.v[0], c.v[1], c.v[2], c.v[3]));
+    } else if constexpr (VEC == 2) {
+        __stcs(reinterpret_cast<float2*>(p), make_float2(c.v[0], c.v[1]));
     } else {
         __stcs(p, c.v[0]);
     }
@@ -80,8 +85,8 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
     const float* __restrict__ ga = HAS_G ? a.g + (size_t)ra * a.ld : nullptr;
     const float* __restrict__ gb = HAS_G ? a.g + (size_t)rb * a.ld : nullptr;
 
-    // columns reachable by whole vectors; the (N mod 4) leftovers are handled at the end
-    const uint32_t nfull = (VEC == 4) ? (a.N & ~3u) : a.N;
+    // columns reachable by whole vectors; the (N mod VEC) leftovers are handled at the end
+    const uint32_t nfull = a.N - a.N % VEC;
     const uint64_t col_tile = (uint64_t)tile * kTileCols;
 
     Chunk<VEC> va[U], vb[U], wa[U], wb[U];
@@ -176,8 +181,8 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
                     for (int q = 0; q < VEC; ++q) c += column_kept(a.col_offset + col[u] + q, a.next_key) ? 1u : 0u;
                 }
             }
-            if constexpr (VEC == 4) {
-                const uint32_t k = nfull + tid;  // the (N mod 4) leftover columns belong to the last tile
+            if constexpr (VEC > 1) {
+                const uint32_t k = nfull + tid;  // the (N mod VEC) leftover columns belong to the last tile
                 if (k < a.N && col_tile <= nfull && nfull < col_tile + kTileCols)
                     c += column_kept(a.col_offset + k, a.next_key) ? 1u : 0u;
             }
@@ -246,8 +251,8 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
         }
     }
 
-    // the last (N mod 4) columns of a row, one thread each
-    if constexpr (VEC == 4) {
+    // the last (N mod VEC) columns of a row, one thread each
+    if constexpr (VEC > 1) {
         const uint32_t ntail = a.N - nfull;
         if (ntail != 0 && tid < ntail && col_tile <= nfull && nfull < col_tile + kTileCols) {
             const uint32_t k = nfull + tid;
@@ -312,9 +317,12 @@ cudaError_t launch_vec(const RoundArgs& a, bool emit, cudaStream_t stream)
 cudaError_t launch_round(const RoundArgs& a, bool emit, cudaStream_t stream)
 {
     if (a.groups.count == 0 || a.tile_count == 0) return cudaSuccess;
-    const bool aligned = (a.ld % 4 == 0) && (reinterpret_cast<uintptr_t>(a.x) % 16 == 0) &&
-                         (a.g == nullptr || reinterpret_cast<uintptr_t>(a.g) % 16 == 0);
-    return aligned ? launch_vec<4>(a, emit, stream) : launch_vec<1>(a, emit, stream);
+    // widest access that every row start allows: 128-bit, else 64-bit, else scalar
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(a.x) | reinterpret_cast<uintptr_t>(a.g) |
+                           (uintptr_t)(a.ld * sizeof(float));
+    if (bits % 16 == 0) return launch_vec<4>(a, emit, stream);
+    if (bits % 8 == 0) return launch_vec<2>(a, emit, stream);
+    return launch_vec<1>(a, emit, stream);
 }
 
 }  // namespace saps
