@@ -252,6 +252,17 @@ SAPS_API int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, 
                     uint64_t T, double keep_frac, const float* lr_list, const int32_t* pairs_list,
                     const double* bandwidth, int32_t* out_pairs_log, void* stream);
 
+/* The same loop with the wire buffer of every round (as saps_round_pack): round r writes its
+ * packed values to out_vals [n, cap] and its kept columns to out_idx [cap] (may be NULL), each
+ * round over the previous one, and its count to out_counts[r] (device, T words).  After the
+ * call the buffers hold the last round's wire data and out_counts the traffic of every round
+ * (Table 1: a worker moves 2 count values per round). */
+SAPS_API int saps_run_rounds_pack(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t t_first,
+                                  uint64_t T, double keep_frac, const float* lr_list,
+                                  const int32_t* pairs_list, const double* bandwidth,
+                                  int32_t* out_pairs_log, float* out_vals, uint32_t* out_idx,
+                                  uint32_t* out_counts, void* stream);
+
 /* ---- host-buffer entry point ----------------------------------------------------------------- */
 
 /* One round on HOST matrices: copies x_host and g_host ([n, N] fp32, row stride N; pinned

@@ -60,6 +60,7 @@ _SIGNATURES = {
     "saps_get_select_state": (_i32, [_vp, _vp, ctypes.POINTER(_u64)]),
     "saps_set_select_state": (_i32, [_vp, _vp, _u64]),
     "saps_run_rounds": (_i32, [_vp, _vp, _vp, _f32, _u64, _u64, _f64, _vp, _vp, _vp, _vp, _vp]),
+    "saps_run_rounds_pack": (_i32, [_vp, _vp, _vp, _f32, _u64, _u64, _f64, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "saps_set_update_order": (_i32, [_vp, _i32]),
     "saps_set_run_ahead": (_i32, [_vp, _i32]),
     "saps_unpack_avg": (_i32, [_vp, _vp, _vp, _vp, _vp, _f64, _vp, _vp]),
@@ -234,6 +235,13 @@ def saps_run_rounds(ctx, x, g, lr, t_first, T, keep_frac, pairs_list=None, bandw
     _check(_lib.saps_run_rounds(ctx, _ptr(x), _ptr(g), lr, t_first, T, keep_frac, _ptr(lr_list),
                                 _ptr(pairs_list), _ptr(bandwidth), _ptr(out_pairs_log), _stream(stream)),
            "saps_run_rounds")
+
+
+def saps_run_rounds_pack(ctx, x, g, lr, t_first, T, keep_frac, out_vals, out_idx, out_counts, pairs_list=None,
+                         bandwidth=None, out_pairs_log=None, stream=None, lr_list=None) -> None:
+    _check(_lib.saps_run_rounds_pack(ctx, _ptr(x), _ptr(g), lr, t_first, T, keep_frac, _ptr(lr_list),
+                                     _ptr(pairs_list), _ptr(bandwidth), _ptr(out_pairs_log), _ptr(out_vals),
+                                     _ptr(out_idx), _ptr(out_counts), _stream(stream)), "saps_run_rounds_pack")
 
 
 SAPS_ORDER_SGD_FIRST = 0

@@ -558,19 +558,29 @@ int saps_set_select_state(saps_ctx* ctx, const int64_t* R, uint64_t last_t)
     return SAPS_OK;
 }
 
-int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t t_first, uint64_t T,
-                    double keep_frac, const float* lr_list, const int32_t* pairs_list,
-                    const double* bandwidth, int32_t* out_pairs_log, void* stream)
+namespace {
+
+// The coordinator's loop (Algorithm 1): for every round, the matching, then the fused round
+// (with the wire buffer when out_vals is given), enqueued back to back without any
+// host-device synchronisation.
+int run_rounds_impl(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t t_first, uint64_t T,
+                    double keep_frac, const float* lr_list, const int32_t* pairs_list, const double* bandwidth,
+                    int32_t* out_pairs_log, float* out_vals, uint32_t* out_idx, uint32_t* out_counts,
+                    cudaStream_t stream)
 {
     int rc = check_round_args(ctx, x, g, lr, t_first, keep_frac);
     if (rc != SAPS_OK) return rc;
     if (pairs_list == nullptr && bandwidth == nullptr) return SAPS_ERR_INVALID;
+    if (t_first + T < t_first) return SAPS_ERR_INVALID;
     if (lr_list != nullptr) {
         if (g == nullptr) return SAPS_ERR_INVALID;
         for (uint64_t r = 0; r < T; ++r)
             if (lr_list[r] != lr_list[r]) return SAPS_ERR_INVALID;
     }
+    const bool emit = out_vals != nullptr;
+    if (emit && out_counts == nullptr) return SAPS_ERR_INVALID;
     const int n = ctx->n;
+    const uint32_t cap = emit ? (uint32_t)saps_pack_capacity(ctx, keep_frac) : 0;
     int32_t chosen[kMaxWorkers];
     for (uint64_t r = 0; r < T; ++r) {
         const uint64_t t = t_first + r;
@@ -585,12 +595,39 @@ int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t 
         rc = check_pairs(n, pairs);
         if (rc != SAPS_OK) return rc;
         if (out_pairs_log != nullptr) std::memcpy(out_pairs_log + r * (uint64_t)n, pairs, sizeof(int32_t) * n);
-        const RowGroups rg = make_groups(n, pairs, g != nullptr);
         const float lr_t = lr_list != nullptr ? lr_list[r] : lr;
-        const RoundArgs a = round_args(ctx, x, g, lr_t, rg, make_key(ctx->seed, t, keep_frac));
-        if (launch_round(a, false, (cudaStream_t)stream) != cudaSuccess) return SAPS_ERR_CUDA;
+        const RowGroups rg = make_groups(n, pairs, g != nullptr || emit);
+        RoundArgs a = round_args(ctx, x, g, lr_t, rg, make_key(ctx->seed, t, keep_frac));
+        if (emit) {
+            rc = prepare_emission(ctx, t, keep_frac, cap, out_idx, out_counts + r, out_vals, stream, &a);
+            if (rc != SAPS_OK) return rc;
+        }
+        if (launch_round(a, emit, stream) != cudaSuccess) {
+            ctx->ahead_valid = false;
+            return SAPS_ERR_CUDA;
+        }
     }
     return SAPS_OK;
+}
+
+}  // namespace
+
+int saps_run_rounds(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t t_first, uint64_t T,
+                    double keep_frac, const float* lr_list, const int32_t* pairs_list,
+                    const double* bandwidth, int32_t* out_pairs_log, void* stream)
+{
+    return run_rounds_impl(ctx, x, g, lr, t_first, T, keep_frac, lr_list, pairs_list, bandwidth, out_pairs_log,
+                           nullptr, nullptr, nullptr, (cudaStream_t)stream);
+}
+
+int saps_run_rounds_pack(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t t_first, uint64_t T,
+                         double keep_frac, const float* lr_list, const int32_t* pairs_list,
+                         const double* bandwidth, int32_t* out_pairs_log, float* out_vals, uint32_t* out_idx,
+                         uint32_t* out_counts, void* stream)
+{
+    if (out_vals == nullptr) return SAPS_ERR_INVALID;
+    return run_rounds_impl(ctx, x, g, lr, t_first, T, keep_frac, lr_list, pairs_list, bandwidth, out_pairs_log,
+                           out_vals, out_idx, out_counts, (cudaStream_t)stream);
 }
 
 namespace {

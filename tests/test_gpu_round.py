@@ -200,10 +200,10 @@ def test_run_rounds_with_given_matchings(sb):
 
 
 def test_run_rounds_with_adaptive_peer_selection(sb):
-    # the ResNet-20-sized configuration, shortened: n=32, N=272,474, keep 0.01, U[1,100] Mb/s
+    # the ResNet-20-sized configuration: n=32, N=272,474, keep 0.01, U[1,100] Mb/s, 100 rounds
     torch = torch_cuda()
     w = synth.WORKLOADS["resnet20"]
-    T = 10
+    T = w.rounds
     x, g = synth.model_and_grad(w)
     B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
     ld = round_up(w.N, 32)
@@ -283,3 +283,46 @@ def test_round_pack_host_entry_point(sb):
     assert (hi.numpy().view(np.uint32)[:wc] == wi[:wc]).all()
     assert_bits_equal(hv.numpy()[:, :wc], wv[:, :wc], "host wire buffer")
     assert_bits_equal(hx.numpy(), want, "host entry point with wire buffer")
+
+
+def test_run_rounds_pack_emits_every_round(sb):
+    # the scheduler with the wire buffer: counts of all rounds, buffers of the last one
+    torch = torch_cuda()
+    w = synth.WORKLOADS["resnet20"]
+    T, p = 12, w.keep_fracs[0]
+    x, g = synth.model_and_grad(w)
+    B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
+    ld = round_up(w.N, 32)
+    dx, dg = DeviceMatrix(x, ld), DeviceMatrix(g, ld)
+    ctx = sb.saps_create_ld(w.n, w.N, ld, w.seed)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.full((w.n, cap), 123.0, dtype=torch.float32, device="cuda")
+    idx = torch.full((cap,), -1, dtype=torch.int32, device="cuda")
+    counts = torch.full((T + 1,), -1, dtype=torch.int32, device="cuda")
+    log = np.zeros((T, w.n), dtype=np.int32)
+    sb.saps_run_rounds_pack(ctx, dx.ptr, dg.ptr, w.lr, 1, T, p, vals, idx, counts, bandwidth=B, out_pairs_log=log)
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    want = x.copy()
+    for t in range(1, T + 1):
+        oracle.sgd(want, g, w.lr)
+        m = oracle.mask(w.seed, t, p, w.N)
+        assert int(counts[t - 1]) == int(m.sum())
+        if t == T:
+            wv, wi, wc = oracle.pack(want, m, cap)
+        oracle.pair_average(want, log[t - 1], m)
+    assert int(counts[T]) == -1
+    assert (idx.cpu().numpy().view(np.uint32)[:wc] == wi[:wc]).all()
+    assert_bits_equal(vals.cpu().numpy()[:, :wc], wv[:, :wc], "last round's wire buffer")
+    assert_bits_equal(dx.host(), want, "scheduler with emission")
+    # Table 1: total traffic of a worker over T rounds is 2 sum_t count_t, about 2 T N / c
+    total = int(counts[:T].sum())
+    phat = oracle.threshold(p) / 2.0 ** 32
+    assert abs(total - T * w.N * phat) < 5 * np.sqrt(T * w.N * phat * (1 - phat))
+    # a given list of matchings works too, and invalid arguments are refused
+    sb.saps_run_rounds_pack(ctx, dx.ptr, dg.ptr, w.lr, T + 1, 2, p, vals, idx, counts, pairs_list=log[:2].copy())
+    torch.cuda.synchronize()
+    rc = sb._lib.saps_run_rounds_pack(ctx, dx.ptr, dg.ptr, w.lr, 1, 2, p, None, None, None, None, None, None, None,
+                                      None, None)
+    assert rc == sb.SAPS_ERR_INVALID
+    sb.saps_destroy(ctx)
