@@ -179,6 +179,14 @@ SAPS_API int saps_unpack_avg(saps_ctx* ctx, float* x, const float* recv_vals, co
                              const uint32_t* count, double keep_frac, const int32_t* pairs,
                              void* stream);
 
+/* The same with an explicit map: worker i averages with row src_rows[i] of recv_vals
+ * (0 <= src_rows[i] < n), or is left alone when src_rows[i] == -1.  This is the form a
+ * row-sharded deployment needs (the workers of one job spread over several GPUs: only the
+ * rows whose peer lives elsewhere receive a buffer).  src_rows: host, n entries. */
+SAPS_API int saps_unpack_avg_rows(saps_ctx* ctx, float* x, const float* recv_vals, const uint32_t* idx,
+                                  const uint32_t* count, double keep_frac, const int32_t* src_rows,
+                                  void* stream);
+
 /* saps_pack for callers that must not allocate device memory.  (The paper has no counterpart:
  * this entry point exists for integration only.)
  *

@@ -64,6 +64,7 @@ _SIGNATURES = {
     "saps_set_update_order": (_i32, [_vp, _i32]),
     "saps_set_run_ahead": (_i32, [_vp, _i32]),
     "saps_unpack_avg": (_i32, [_vp, _vp, _vp, _vp, _vp, _f64, _vp, _vp]),
+    "saps_unpack_avg_rows": (_i32, [_vp, _vp, _vp, _vp, _vp, _f64, _vp, _vp]),
     "saps_consensus_distance": (_i32, [_vp, _vp, _vp, _vp]),
     "saps_comm_stats": (_i32, [_vp, _vp, _vp, _u64, _f64, _vp]),
     "saps_debug_inject": (_i32, [_vp, _u32, _u32]),
@@ -259,6 +260,11 @@ def saps_set_run_ahead(ctx, enabled: bool) -> None:
 def saps_unpack_avg(ctx, x, recv_vals, idx, count, keep_frac, pairs=None, stream=None) -> None:
     _check(_lib.saps_unpack_avg(ctx, _ptr(x), _ptr(recv_vals), _ptr(idx), _ptr(count), keep_frac,
                                 None if pairs is None else _pairs(pairs), _stream(stream)), "saps_unpack_avg")
+
+
+def saps_unpack_avg_rows(ctx, x, recv_vals, idx, count, keep_frac, src_rows, stream=None) -> None:
+    _check(_lib.saps_unpack_avg_rows(ctx, _ptr(x), _ptr(recv_vals), _ptr(idx), _ptr(count), keep_frac,
+                                     _pairs(src_rows), _stream(stream)), "saps_unpack_avg_rows")
 
 
 def saps_consensus_distance(ctx, x, out, stream=None) -> None:

@@ -289,19 +289,13 @@ int saps_set_update_order(saps_ctx* ctx, int order)
     return SAPS_OK;
 }
 
-int saps_unpack_avg(saps_ctx* ctx, float* x, const float* recv_vals, const uint32_t* idx, const uint32_t* count,
-                    double keep_frac, const int32_t* pairs, void* stream)
+namespace {
+
+int unpack_avg_impl(saps_ctx* ctx, float* x, const float* recv_vals, const uint32_t* idx, const uint32_t* count,
+                    double keep_frac, const uint8_t* src, cudaStream_t stream)
 {
-    if (ctx == nullptr || x == nullptr || recv_vals == nullptr || idx == nullptr || count == nullptr ||
-        !valid_frac(keep_frac))
-        return SAPS_ERR_INVALID;
     UnpackArgs a;
-    if (pairs != nullptr) {
-        const int rc = check_pairs(ctx->n, pairs);
-        if (rc != SAPS_OK) return rc;
-    }
-    for (int i = 0; i < ctx->n; ++i)
-        a.src[i] = pairs == nullptr ? (uint8_t)i : (pairs[i] == i ? kNoPeer : (uint8_t)pairs[i]);
+    std::memcpy(a.src, src, kMaxWorkers);
     a.x = x;
     a.ld = (size_t)ctx->ld;
     a.n = ctx->n;
@@ -311,7 +305,39 @@ int saps_unpack_avg(saps_ctx* ctx, float* x, const float* recv_vals, const uint3
     a.count = count;
     a.col_offset = (uint32_t)ctx->col_offset;
     a.N = (uint32_t)ctx->N;
-    return launch_unpack_avg(a, (cudaStream_t)stream) == cudaSuccess ? SAPS_OK : SAPS_ERR_CUDA;
+    return launch_unpack_avg(a, stream) == cudaSuccess ? SAPS_OK : SAPS_ERR_CUDA;
+}
+
+}  // namespace
+
+int saps_unpack_avg(saps_ctx* ctx, float* x, const float* recv_vals, const uint32_t* idx, const uint32_t* count,
+                    double keep_frac, const int32_t* pairs, void* stream)
+{
+    if (ctx == nullptr || x == nullptr || recv_vals == nullptr || idx == nullptr || count == nullptr ||
+        !valid_frac(keep_frac))
+        return SAPS_ERR_INVALID;
+    if (pairs != nullptr) {
+        const int rc = check_pairs(ctx->n, pairs);
+        if (rc != SAPS_OK) return rc;
+    }
+    uint8_t src[kMaxWorkers] = {};
+    for (int i = 0; i < ctx->n; ++i)
+        src[i] = pairs == nullptr ? (uint8_t)i : (pairs[i] == i ? kNoPeer : (uint8_t)pairs[i]);
+    return unpack_avg_impl(ctx, x, recv_vals, idx, count, keep_frac, src, (cudaStream_t)stream);
+}
+
+int saps_unpack_avg_rows(saps_ctx* ctx, float* x, const float* recv_vals, const uint32_t* idx,
+                         const uint32_t* count, double keep_frac, const int32_t* src_rows, void* stream)
+{
+    if (ctx == nullptr || x == nullptr || recv_vals == nullptr || idx == nullptr || count == nullptr ||
+        src_rows == nullptr || !valid_frac(keep_frac))
+        return SAPS_ERR_INVALID;
+    uint8_t src[kMaxWorkers] = {};
+    for (int i = 0; i < ctx->n; ++i) {
+        if (src_rows[i] < -1 || src_rows[i] >= ctx->n) return SAPS_ERR_INVALID;
+        src[i] = src_rows[i] < 0 ? kNoPeer : (uint8_t)src_rows[i];
+    }
+    return unpack_avg_impl(ctx, x, recv_vals, idx, count, keep_frac, src, (cudaStream_t)stream);
 }
 
 int saps_consensus_distance(saps_ctx* ctx, const float* x, double* out, void* stream)

@@ -191,3 +191,49 @@ def test_bounded_wait_reports_a_timeout_instead_of_hanging(sb):
     assert int(count[0]) == wc
     assert_bits_equal(vals.cpu().numpy()[:, :wc], wv[:, :wc], "pack after a timed-out call")
     sb.saps_destroy(ctx)
+
+
+def test_row_sharded_round_emulated_on_one_gpu(sb):
+    # Two "ranks" of 4 workers each, run one after the other on this GPU; the transfer between
+    # them is a device copy of the packed rows.  The result must equal the single-context round.
+    torch = torch_cuda()
+    from paper_2002_09692_b200.row_sharded import RowShardedGossip
+    world, per_rank, N, p, lr, seed = 2, 4, 30_000, 0.05, 0.05, 33
+    n = world * per_rank
+    ld = round_up(N, 32)
+    x = synth.gaussian_matrix(n, N, 1.0, 33, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, 33, 1)
+    rng = synth.matching_rng(33)
+    ranks = [RowShardedGossip(r, world, per_rank, N, ld, seed) for r in range(world)]
+    dxs = [DeviceMatrix(np.ascontiguousarray(x[r * per_rank:(r + 1) * per_rank]), ld) for r in range(world)]
+    dgs = [DeviceMatrix(np.ascontiguousarray(g[r * per_rank:(r + 1) * per_rank]), ld) for r in range(world)]
+    cap = sb.saps_pack_capacity(ranks[0].ctx, p)
+    bufs = [dict(vals=torch.zeros(per_rank, cap, device="cuda"), recv=torch.zeros(per_rank, cap, device="cuda"),
+                 idx=torch.zeros(cap, dtype=torch.int32, device="cuda"),
+                 count=torch.zeros(1, dtype=torch.int32, device="cuda")) for _ in range(world)]
+    want = x.copy()
+    crossed = 0
+    for t in range(1, 6):
+        pairs = synth.random_perfect_matching(n, rng)
+        plans = [ranks[r].local_step(dxs[r].ptr, dgs[r].ptr, lr, pairs, t, p, bufs[r]["vals"], bufs[r]["idx"],
+                                     bufs[r]["count"]) for r in range(world)]
+        for r in range(world):                              # the wire: each packed row goes to its peer's rank
+            for row, peer, _tag in plans[r].transfers:
+                j = int(pairs[r * per_rank + row])
+                bufs[peer]["recv"][j - peer * per_rank].copy_(bufs[r]["vals"][row])
+                crossed += 1
+        for r in range(world):
+            ranks[r].merge(dxs[r].ptr, plans[r], bufs[r]["recv"], bufs[r]["idx"], bufs[r]["count"], p)
+        oracle.gossip_round(want, g, lr, pairs, seed, t, p)
+    torch.cuda.synchronize()
+    assert crossed > 0
+    got = np.concatenate([d.host() for d in dxs], axis=0)
+    assert_bits_equal(got, want, "row-sharded round")
+    assert all(d.canaries_intact() for d in dxs)
+    for rk in ranks:
+        rk.close()
+    # the explicit row map refuses rows outside the context
+    ctx = sb.saps_create(4, 100, 0)
+    assert sb._lib.saps_unpack_avg_rows(ctx, 0x1000, 0x1000, 0x1000, 0x1000, 0.5, sb._pairs([0, 1, 2, 4]), None) \
+        == sb.SAPS_ERR_INVALID
+    sb.saps_destroy(ctx)

@@ -80,3 +80,59 @@ def test_two_ranks_gloo():
     assert res[0][3] == 0 and res[1][3] == res[0][2]                    # exclusive scan of the counts
     assert res[0][4] == res[1][4] == int(full.sum()) == res[0][2] + res[1][2]
     assert res[0][5] == res[1][5] == 11.0                               # the slowest rank's time
+
+
+# ---- row-sharded deployment: planning and the exchange step, on CPU ranks ---------------------
+
+def test_plan_row_exchange_splits_a_matching():
+    from paper_2002_09692_b200.row_sharded import plan_row_exchange
+    pairs = [1, 0, 5, 6, 7, 2, 3, 4]                     # 8 workers, 2 ranks of 4
+    p0 = plan_row_exchange(pairs, 0, 2, 4)
+    p1 = plan_row_exchange(pairs, 1, 2, 4)
+    assert p0.local_pairs == (1, 0, 2, 3) and p0.src_rows == (-1, -1, 2, 3)
+    assert p0.transfers == ((2, 1, 2), (3, 1, 3))
+    assert p1.local_pairs == (3, 1, 2, 0) and p1.src_rows == (-1, 1, 2, -1)
+    assert p1.transfers == ((1, 0, 2), (2, 0, 3))        # same tags as on rank 0
+    with pytest.raises(ValueError):
+        plan_row_exchange([1, 2, 0, 3], 0, 2, 2)
+
+
+def _row_worker(rank, world, port, results):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        from paper_2002_09692_b200.row_sharded import exchange_rows, plan_row_exchange
+        per_rank, cap = 4, 6
+        rng = np.random.default_rng(5)
+        ok = True
+        for _ in range(5):
+            pairs = synth.random_perfect_matching(world * per_rank, rng)     # same stream on both ranks
+            plan = plan_row_exchange(pairs, rank, world, per_rank)
+            send = torch.arange(per_rank * cap, dtype=torch.float32).reshape(per_rank, cap) + 1000.0 * rank
+            recv = torch.full((per_rank, cap), -1.0)
+            exchange_rows(send, recv, plan)
+            for r in range(per_rank):
+                j = int(pairs[rank * per_rank + r])
+                if j // per_rank == rank:
+                    ok &= bool((recv[r] == -1.0).all())                      # nothing arrives for local pairs
+                else:
+                    want = torch.arange(cap, dtype=torch.float32) + (j % per_rank) * cap + 1000.0 * (j // per_rank)
+                    ok &= bool((recv[r] == want).all())                      # the peer's row, whole
+        results[rank] = ok
+    finally:
+        dist.destroy_process_group()
+
+
+def test_row_exchange_two_ranks_gloo():
+    world = 2
+    ctx = mp.get_context("spawn")
+    with ctx.Manager() as mgr:
+        results = mgr.dict()
+        port = _free_port()
+        procs = [ctx.Process(target=_row_worker, args=(r, world, port, results)) for r in range(world)]
+        for pr in procs:
+            pr.start()
+        for pr in procs:
+            pr.join(120)
+            assert pr.exitcode == 0
+        assert results[0] is True and results[1] is True
