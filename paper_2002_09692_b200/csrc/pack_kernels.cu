@@ -196,49 +196,49 @@ __global__ void __launch_bounds__(kThreads) mask_count_kernel(uint32_t N, uint32
     if (lane == 0) tile_cnt[tile] = cnt;
 }
 
-// Exclusive prefix of the tile counts, the total and the overflow check: one block walks the
-// list in chunks of its size (a few chunks for tens of millions of columns).
+// Exclusive prefix of the tile counts, the total and the overflow check, by one block: every
+// thread owns a contiguous run of tiles (a handful for tens of millions of columns), sums it,
+// the block scans the 1024 sums once, and every thread writes the prefixes of its run.
 constexpr int kScanThreads = 1024;
 __global__ void __launch_bounds__(kScanThreads) tile_scan_kernel(const uint32_t* __restrict__ tile_cnt,
                                                                  uint32_t ntiles, uint32_t* __restrict__ tile_excl,
                                                                  uint32_t* out_count, uint32_t cap, int* status)
 {
     __shared__ uint32_t s_warp[kScanThreads / 32];
-    __shared__ uint32_t s_carry;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) s_carry = 0;
+    const uint32_t per = (ntiles + kScanThreads - 1) / kScanThreads;
+    const uint64_t lo64 = (uint64_t)tid * per;
+    const uint32_t lo = lo64 < ntiles ? (uint32_t)lo64 : ntiles;
+    const uint32_t hi = lo64 + per < ntiles ? (uint32_t)(lo64 + per) : ntiles;
+    uint32_t mine = 0;
+    for (uint32_t i = lo; i < hi; ++i) mine += tile_cnt[i];
+    uint32_t inc = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += o;
+    }
+    if (lane == 31) s_warp[warp] = inc;
     __syncthreads();
-    for (uint32_t base = 0; base < ntiles; base += kScanThreads) {
-        const uint32_t i = base + tid;
-        const uint32_t c = i < ntiles ? tile_cnt[i] : 0u;
-        uint32_t inc = c;
+    if (warp == 0) {
+        uint32_t w = s_warp[lane];
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-            if (lane >= d) inc += o;
+            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, w, d);
+            if (lane >= d) w += o;
         }
-        if (lane == 31) s_warp[warp] = inc;
-        __syncthreads();
-        if (warp == 0) {
-            uint32_t w = s_warp[lane];
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, w, d);
-                if (lane >= d) w += o;
-            }
-            s_warp[lane] = w;  // inclusive over warps
-        }
-        __syncthreads();
-        const uint32_t carry = s_carry;
-        const uint32_t before = carry + (warp ? s_warp[warp - 1] : 0u) + inc - c;
-        if (i < ntiles) tile_excl[i] = before;
-        __syncthreads();
-        if (tid == kScanThreads - 1) s_carry = carry + s_warp[kScanThreads / 32 - 1];
-        __syncthreads();
+        s_warp[lane] = w;  // inclusive over warps
     }
-    if (tid == 0) {
-        if (out_count != nullptr) *out_count = s_carry;
-        if (s_carry > cap) atomicCAS(status, 0, -4 /* SAPS_ERR_OVERFLOW */);
+    __syncthreads();
+    uint32_t run = (warp ? s_warp[warp - 1] : 0u) + inc - mine;
+    for (uint32_t i = lo; i < hi; ++i) {
+        tile_excl[i] = run;
+        run += tile_cnt[i];
+    }
+    if (tid == kScanThreads - 1) {
+        const uint32_t total = s_warp[kScanThreads / 32 - 1];
+        if (out_count != nullptr) *out_count = total;
+        if (total > cap) atomicCAS(status, 0, -4 /* SAPS_ERR_OVERFLOW */);
     }
 }
 

@@ -89,6 +89,10 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
     const uint32_t nfull = a.N - a.N % VEC;
     const uint64_t col_tile = (uint64_t)tile * kTileCols;
 
+    // the tile's rank offset is asked for first, so that its latency hides under the model loads
+    uint32_t excl = 0;
+    if constexpr (EMIT) excl = __ldg(a.tile_excl + tile);
+
     Chunk<VEC> va[U], vb[U], wa[U], wb[U];
     bool inb[U];
     uint32_t col[U];
@@ -128,7 +132,6 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
 
     uint32_t rank[U];       // EMIT only: rank of this thread's first kept column
     uint32_t total = 0;     // EMIT only: kept columns in the vector part of the tile
-    uint32_t excl = 0;
     if constexpr (EMIT) {
         __shared__ uint32_t s_warp[U][kWarps];
         const int lane = tid & 31, warp = tid >> 5;
@@ -141,7 +144,6 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
             if (lane == 31) s_warp[u][warp] = inc;
         }
         __syncthreads();
-        excl = a.tile_excl[tile];
         uint32_t running = excl;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
