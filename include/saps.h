@@ -34,9 +34,13 @@
  *     round; it must be an involution (pairs[pairs[i]] == i).
  *   - fp32 arithmetic is IEEE round-to-nearest, one rounding per operation, never fused:
  *     a = x - fl(lr * g);  avg = fl(0.5f * fl(a_i + a_j)).  Subnormals are kept.
- *   - The context owns a small device scratch area (tile states of the compaction scan,
- *     a status word).  It is allocated by the first call that needs it, on the device that
- *     is current then; that first call must not happen inside a stream capture.
+ *   - The context owns small device scratch areas, each allocated by the first call that
+ *     needs it, on the device that is current then (so such a first call must not happen
+ *     inside a stream capture): the status word and the tile states of the compaction scan
+ *     (16 + 12 ceil(N/2048) bytes; saps_pack and every emitting entry point), the per-tile
+ *     counts and prefixes of the emitting round (12 ceil(N/2048) bytes), the partial sums of
+ *     saps_consensus_distance (8 ceil(N/2048) bytes).  saps_round, saps_run_rounds,
+ *     saps_mask, saps_unpack_avg* and saps_pack_noalloc allocate nothing.
  *   - Calls on one context must not overlap on the GPU (use one stream, or order streams
  *     with events): they share the scratch area.
  */
