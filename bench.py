@@ -66,7 +66,9 @@ class ClockSampler:
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_id):
+        """gpu_id: what `nvidia-smi -i` accepts (an index or a "GPU-<uuid>" string)."""
+        gpu_index = gpu_id
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.proc = None
         try:
@@ -239,7 +241,11 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
+    try:        # the CUDA ordinal need not be nvidia-smi's index (CUDA_VISIBLE_DEVICES): go by UUID
+        smi_id = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        smi_id = local
+    sampler = ClockSampler(smi_id)
     time.sleep(0.3)
     barrier()
     ev_start.record(stream)
@@ -290,6 +296,20 @@ def run_ours(args):
             "traffic": None if NCU_TRAFFIC_BYTES_PER_ELEMENT is None else NCU_TRAFFIC_BYTES_PER_ELEMENT * n * N,
         },
     }
+
+    # the same K steps a few more times (context: spread of the measurement; `value` is the first)
+    repeats = []
+    for _ in range(4):
+        barrier()
+        ev_start.record(stream)
+        for k in range(K):
+            step(t)
+            t += 1
+        ev_stop.record(stream)
+        barrier()
+        repeats.append(sharding.max_over_ranks(ev_start.elapsed_time(ev_stop)) / K)
+    result["repeat_ms_per_step"] = {"all": [ms_per_step] + repeats, "median": statistics.median([ms_per_step] + repeats),
+                                    "best": min([ms_per_step] + repeats)}
 
     # the other entry points of the path, timed alone on the same resident inputs (context only)
     def timed(fn, reps=20):
