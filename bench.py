@@ -33,7 +33,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per worker-parameter of the fused round kernel, from the ncu
 # capture of that kernel on a smaller workload (summary under profiles/; traffic grows in proportion
 # to n*N).  Set to None whenever round_kernels.cu changes until the counters are retaken.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = 11.787
+NCU_TRAFFIC_BYTES_PER_ELEMENT = 11.790
 
 
 def parse_args():
