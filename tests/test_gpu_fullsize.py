@@ -136,3 +136,65 @@ def test_gpt2s_sampled_rows(sb):
     rows = {5, int(pairs[5])}
     _sampled_round(sb, torch, w, 0.01, 1, pairs, rows, golden=_golden_count(0, 1, w.N, 0.01))
     torch.cuda.empty_cache()
+
+
+def test_largest_column_count(sb):
+    # N just below 2^32 (the largest the 32-bit column index allows), ragged (N mod 4 = 3),
+    # two workers, pure gossip with emission.  Checked against the oracle's hash on sampled and
+    # on the very last columns, and by device-side invariants on all 8.6e9 elements.
+    torch = torch_cuda()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 100 * 2 ** 30:
+        pytest.skip("needs about 100 GB of free device memory")
+    n, N, ld, seed, t, p = 2, 2 ** 32 - 5, 2 ** 32, 7, 3, 1e-4
+    x = torch.empty(n, ld, dtype=torch.float32, device="cuda").normal_(0.0, 1.0)
+    x0 = x.clone()
+    ctx = sb.saps_create_ld(n, N, ld, seed)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    count = torch.zeros(1, dtype=torch.int32, device="cuda")
+    bits = torch.zeros(2 ** 27, dtype=torch.int32, device="cuda")
+    sb.saps_mask(ctx, t, p, bits)
+    sb.saps_round_pack(ctx, x, None, 0.0, [1, 0], t, p, vals, idx, count)
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    c = int(count.cpu().numpy().view(np.uint32)[0])
+    thr = oracle.threshold(p)
+    phat = thr / 2.0 ** 32
+    assert abs(c - N * phat) < 5 * np.sqrt(N * phat * (1 - phat))
+    # the bitmap agrees with the count, and has nothing at or beyond N
+    words = bits.cpu().numpy().view(np.uint32)
+    assert int(np.unpackbits(words.view(np.uint8)).sum(dtype=np.int64)) == c
+    assert words[-1] >> 27 == 0                                   # columns 2^32-5 .. 2^32-1 do not exist
+    # index list: strictly ascending, every sampled entry is a kept column by the oracle's hash
+    cols = idx[:c].cpu().numpy().view(np.uint32).astype(np.int64)
+    assert (np.diff(cols) > 0).all() and cols[-1] < N
+    k0, k1 = oracle.round_key(seed, t)
+    rng = np.random.default_rng(0)
+    for r in list(rng.integers(0, c, 300)) + [0, c - 1]:
+        assert oracle.hash_k(int(cols[r]), k0, k1) < thr
+    # the last 2^17 columns, one by one: exactly the oracle's kept set (32-bit wrap would show here)
+    lo = N - 2 ** 17
+    want_tail = [k for k in range(lo, N) if oracle.hash_k(k, k0, k1) < thr]
+    assert list(cols[cols >= lo]) == want_tail
+    # wire buffer = the senders' values at the kept columns
+    gather = torch.from_numpy(cols).cuda()
+    assert torch.equal(vals[:, :c], x0[:, gather])
+    # the model: kept columns hold the pair mean on both workers, everything else is untouched
+    mean = 0.5 * (x0[0, gather] + x0[1, gather])
+    assert torch.equal(x[0, gather], mean) and torch.equal(x[1, gather], mean)
+    x0[:, gather] = x[:, gather]
+    assert torch.equal(x, x0)                                     # includes the padding columns
+    # the standalone compaction (two million look-back tiles) finds the same columns
+    vals2 = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
+    idx2 = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    count2 = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sb.saps_pack(ctx, x, t, p, vals2, idx2, count2)
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    assert int(count2.cpu().numpy().view(np.uint32)[0]) == c and torch.equal(idx2[:c], idx[:c])
+    assert torch.equal(vals2[:, :c], x[:, gather])
+    sb.saps_destroy(ctx)
+    del x, x0
+    torch.cuda.empty_cache()
