@@ -37,10 +37,9 @@ def build(force: bool = False) -> Path:
 _lib = None
 
 
-def _c():
-    global _lib
-    if _lib is None:
-        lib = ctypes.CDLL(str(build()))
+def _bind(lib):
+    """Declare the C signatures on a loaded oracle library."""
+    if True:
         u32, u64, i32 = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int
         vp, dbl, f32 = ctypes.c_void_p, ctypes.c_double, ctypes.c_float
         lib.orc_mix.restype = u32
@@ -67,7 +66,13 @@ def _c():
         lib.orc_unpack_avg.argtypes = [i32, u64, vp, vp, u64, vp, u64]
         lib.orc_consensus_distance.restype = dbl
         lib.orc_consensus_distance.argtypes = [i32, u64, vp]
-        _lib = lib
+    return lib
+
+
+def _c():
+    global _lib
+    if _lib is None:
+        _lib = _bind(ctypes.CDLL(str(build())))
     return _lib
 
 

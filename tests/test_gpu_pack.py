@@ -243,3 +243,19 @@ def test_round_pack_sequence_with_scan_run_ahead(sb, prefetch):
         assert_bits_equal(dx.host(), want, f"model step {step}")
     assert sb.saps_status(ctx) == 0
     sb.saps_destroy(ctx)
+
+
+def test_threshold_comparison_is_strict_on_the_gpu(sb):
+    # a column whose hash equals the threshold is dropped; one more and it is kept
+    torch = torch_cuda()
+    seed, t, N = 12, 34, 100_001
+    k0, k1 = oracle.round_key(seed, t)
+    ctx = sb.saps_create(2, N, seed)
+    bits = torch.zeros(round_up(N, 32) // 32, dtype=torch.int32, device="cuda")
+    for k in (0, 1, 77, 4095, 100_000):
+        h = oracle.hash_k(k, k0, k1)
+        for thr, want in ((h, 0), (h + 1, 1)):
+            sb.saps_mask(ctx, t, thr / 2.0 ** 32, bits)
+            word = int(bits[k >> 5].cpu().numpy().view(np.uint32))
+            assert (word >> (k & 31)) & 1 == want
+    sb.saps_destroy(ctx)

@@ -135,3 +135,16 @@ def test_traffic_closed_form():
     total = sum(int(oracle.mask(1, t, p, N).sum(dtype=np.int64)) for t in range(1, T + 1))
     sigma = math.sqrt(T * N * phat * (1 - phat))
     assert abs(2 * total - 2 * T * N * phat) < 2 * 5.0 * sigma
+
+
+def test_threshold_comparison_is_strict():
+    # keep(k) is "hash < threshold": with the threshold set to a column's own hash value that
+    # column is dropped, one more and it is kept (floor(keep_frac 2^32) is exact for h / 2^32)
+    seed, t = 12, 34
+    k0, k1 = oracle.round_key(seed, t)
+    for k in (0, 1, 77, 4095, 100_000):
+        h = oracle.hash_k(k, k0, k1)
+        assert oracle.threshold(h / 2.0 ** 32) == h
+        assert oracle.mask(seed, t, h / 2.0 ** 32, k + 1)[k] == 0
+        if h + 1 <= 2 ** 32:
+            assert oracle.mask(seed, t, (h + 1) / 2.0 ** 32, k + 1)[k] == 1
