@@ -263,3 +263,16 @@ def test_bottleneck_threshold_with_missing_links_and_odd_n():
     bigger = [v for v in np.unique(S) if v > theta]
     assert all(len(ps.maximum_matching(S >= v)) < 2 for v in bigger)
     assert ps.bottleneck_threshold(np.zeros((4, 4))) == 0.0
+
+
+def test_record_round_stamps_the_round():
+    # the timestamp matrix records the exchange of round t (Section II-C): an edge used in
+    # round t stays "recently connected" for exactly T_thres rounds
+    R = ps.new_timestamps(4)
+    ps.record_round(R, [1, 0, 3, 2], 7)
+    assert R[0, 1] == R[1, 0] == R[2, 3] == R[3, 2] == 7
+    assert R[0, 2] == ps.NEVER and R[0, 0] == ps.NEVER
+    T = 5
+    assert ps.recent_graph(R, 7 + T - 1, T)[0, 1] and not ps.recent_graph(R, 7 + T, T)[0, 1]
+    ps.record_round(R, [0, 2, 1, 3], 9)                  # workers 0 and 3 sit this round out
+    assert R[1, 2] == R[2, 1] == 9 and R[0, 1] == 7 and R[0, 0] == ps.NEVER
