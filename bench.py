@@ -30,10 +30,11 @@ if ROOT not in sys.path:
 METRIC = "gossip_rounds_per_s"
 UNIT = "rounds/s"
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (read + write) per worker-parameter of the fused round kernel, from the ncu
-# capture of that kernel on a smaller workload (summary under profiles/; traffic grows in proportion
-# to n*N).  Set to None whenever round_kernels.cu changes until the counters are retaken.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = 11.790
+# DRAM bytes (read + write) per worker-parameter of the fused round kernel, from ncu's
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch on the vgg16 workload (summary
+# under profiles/; for other workloads the traffic is scaled in proportion to n*N).  Set to
+# None whenever round_kernels.cu changes until the counters are retaken.
+NCU_TRAFFIC_BYTES_PER_ELEMENT = 5_620_820_736 / (32 * 14_728_266)
 
 
 def parse_args():
