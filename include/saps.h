@@ -285,6 +285,10 @@ SAPS_API int saps_run_rounds_pack(saps_ctx* ctx, float* x, const float* g, float
 SAPS_API int saps_round_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
                     const int32_t* pairs, uint64_t t, double keep_frac, float* d_x, float* d_g);
 
+/* In both host-buffer entry points x_host may be NULL: the model then stays resident in d_x
+ * from call to call (as in training, where the weights live on the GPU) and only the
+ * gradients travel in and, for saps_round_pack_host, the wire buffer travels out. */
+
 /* The same with the wire buffer of step 3 (as saps_round_pack): out_vals_host [n, cap],
  * out_idx_host [cap] or NULL, out_count_host (one word) are HOST buffers filled before the
  * call returns; d_vals [n, cap], d_idx [cap], d_count are device staging (d_idx may be NULL

@@ -695,7 +695,8 @@ int ensure_lanes(saps_ctx* ctx)
 int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr, const int32_t* pairs,
                     uint64_t t, double keep_frac, float* d_x, float* d_g, const HostPack* pack)
 {
-    int rc = check_round_args(ctx, x_host, g_host, lr, t, keep_frac);
+    // x_host == NULL: the model stays resident in d_x; only the gradients travel in
+    int rc = check_round_args(ctx, d_x, g_host, lr, t, keep_frac);
     if (rc != SAPS_OK) return rc;
     if (d_x == nullptr || (g_host != nullptr && d_g == nullptr)) return SAPS_ERR_INVALID;
     if (pack != nullptr && (pack->vals_host == nullptr || pack->count_host == nullptr || pack->d_vals == nullptr ||
@@ -731,8 +732,9 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
         const uint64_t c1 = c0 + (uint64_t)tc * kTileCols < N ? c0 + (uint64_t)tc * kTileCols : N;
         const size_t width = (size_t)(c1 - c0) * sizeof(float);
         cudaStream_t s = ctx->lane_stream[lane];
-        failed |= cudaMemcpy2DAsync(d_x + c0, ld_dev * sizeof(float), x_host + c0, N * sizeof(float), width, n,
-                                    cudaMemcpyHostToDevice, s) != cudaSuccess;
+        if (x_host != nullptr)
+            failed |= cudaMemcpy2DAsync(d_x + c0, ld_dev * sizeof(float), x_host + c0, N * sizeof(float), width, n,
+                                        cudaMemcpyHostToDevice, s) != cudaSuccess;
         if (g_host != nullptr)
             failed |= cudaMemcpy2DAsync(d_g + c0, ld_dev * sizeof(float), g_host + c0, N * sizeof(float), width,
                                         n, cudaMemcpyHostToDevice, s) != cudaSuccess;
@@ -740,8 +742,9 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
         a.tile_begin = tb;
         a.tile_count = tc;
         failed |= launch_round(a, emit, s) != cudaSuccess;
-        failed |= cudaMemcpy2DAsync(x_host + c0, N * sizeof(float), d_x + c0, ld_dev * sizeof(float), width, n,
-                                    cudaMemcpyDeviceToHost, s) != cudaSuccess;
+        if (x_host != nullptr)
+            failed |= cudaMemcpy2DAsync(x_host + c0, N * sizeof(float), d_x + c0, ld_dev * sizeof(float), width, n,
+                                        cudaMemcpyDeviceToHost, s) != cudaSuccess;
     }
     if (emit && !failed) {
         // the wire buffer is complete once every lane has run its chunks

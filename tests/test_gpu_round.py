@@ -283,6 +283,14 @@ def test_round_pack_host_entry_point(sb):
     assert (hi.numpy().view(np.uint32)[:wc] == wi[:wc]).all()
     assert_bits_equal(hv.numpy()[:, :wc], wv[:, :wc], "host wire buffer")
     assert_bits_equal(hx.numpy(), want, "host entry point with wire buffer")
+    # model resident on the device (x_host = NULL): only g goes in, the wire buffer comes out
+    ctx = sb.saps_create(n, N, 52)
+    d_x.view(n, ld)[:, :N].copy_(torch.from_numpy(x))
+    sb.saps_round_pack_host(ctx, None, hg, 0.05, pairs, 4, p, d_x, d_g, hv, hi, hc, d_v, d_i, d_c)
+    assert int(hc[0]) == wc
+    assert_bits_equal(hv.numpy()[:, :wc], wv[:, :wc], "host wire buffer, resident model")
+    assert_bits_equal(d_x.view(n, ld)[:, :N].cpu().numpy(), want, "resident model after the round")
+    sb.saps_destroy(ctx)
 
 
 def test_run_rounds_pack_emits_every_round(sb):
