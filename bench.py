@@ -30,11 +30,39 @@ if ROOT not in sys.path:
 METRIC = "gossip_rounds_per_s"
 UNIT = "rounds/s"
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (read + write) per worker-parameter of the fused round kernel, from ncu's
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch on the vgg16 workload (summary
-# under profiles/; for other workloads the traffic is scaled in proportion to n*N).  Set to
-# None whenever round_kernels.cu changes until the counters are retaken.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = 5_620_820_736 / (32 * 14_728_266)
+L2_BYTES = 126e6
+# DRAM bytes (read + write) of ONE launch of the fused round kernel, from ncu's
+# dram__bytes_read.sum + dram__bytes_write.sum on the workload below (summary:
+# profiles/round_kernel_vgg16_traffic_ncu.md).  The figure is only reported for that workload
+# and only while the kernel's sources still hash to what was captured; otherwise null.
+NCU_TRAFFIC = {
+    "workload": "vgg16", "keep_frac": 0.01, "bytes_per_launch": 5_620_820_736,
+    "source": "profiles/round_kernel_vgg16_traffic_ncu.md",
+    "kernel_sources": ("paper_2002_09692_b200/csrc/round_kernels.cu", "paper_2002_09692_b200/csrc/mask_hash.cuh"),
+    "kernel_sources_sha256": "UNSET",
+}
+ORACLE_MAX_COLUMNS = 1 << 24          # the CPU oracle runs full width up to this many columns
+
+
+def kernel_sources_hash():
+    import hashlib
+    h = hashlib.sha256()
+    for rel in NCU_TRAFFIC["kernel_sources"]:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def ncu_traffic(workload, keep_frac):
+    """The captured DRAM traffic per launch, or None when it does not describe this run."""
+    if workload != NCU_TRAFFIC["workload"] or keep_frac != NCU_TRAFFIC["keep_frac"]:
+        return None
+    try:
+        if kernel_sources_hash() != NCU_TRAFFIC["kernel_sources_sha256"]:
+            return None
+    except OSError:
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"]
 
 
 def parse_args():
@@ -46,9 +74,11 @@ def parse_args():
     ap.add_argument("--workload", default="vgg16")
     ap.add_argument("--keep-frac", type=float, default=0.01)
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--cpu-rounds", type=int, default=4)
+    ap.add_argument("--cpu-rounds", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-verify", action="store_true")
+    ap.add_argument("--no-small-loop", action="store_true")
     return ap.parse_args()
 
 
@@ -132,6 +162,17 @@ def oracle_step(oracle, ps, x, g, w, B, R, t, keep_frac, b_thres, t_thres, cap):
     oracle.pair_average(x, np.asarray(pairs, dtype=np.int32), m)
 
 
+def oracle_sample(w):
+    """Columns the oracle runs on per step: the whole model when it has at most
+    ORACLE_MAX_COLUMNS columns (the benchmark's default workload has), else the first
+    ORACLE_MAX_COLUMNS, with rounds/s scaled in proportion."""
+    cols = min(w.N, ORACLE_MAX_COLUMNS)
+    if cols == w.N:
+        return cols, f"all {w.N} columns of all {w.n} workers per step (nothing scaled)"
+    return cols, (f"first {cols} of {w.N} columns of all {w.n} workers per step; "
+                  f"rounds/s scaled by {cols}/{w.N}")
+
+
 def run_reference(args):
     rank, world, _ = dist_env()
     if rank != 0:
@@ -142,7 +183,7 @@ def run_reference(args):
     from oracle import peer_selection as ps
     from paper_2002_09692_b200 import synth
     w = synth.WORKLOADS[args.workload]
-    cols = min(w.N, 1 << 21)           # bounded sample: the first `cols` columns of every worker
+    cols, sample = oracle_sample(w)
     x = synth.gaussian_matrix(w.n, cols, w.x_std, w.seed, 0)
     g = synth.gaussian_matrix(w.n, cols, w.g_std, w.seed, 1)
     B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
@@ -160,16 +201,33 @@ def run_reference(args):
     dt = time.perf_counter() - t0
     ms = dt / args.steps * 1e3
     value = (cols / w.N) / (dt / args.steps)
-    sample = f"first {cols} of {w.N} columns of all {w.n} workers per step; rounds/s scaled by {cols}/{w.N}"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{w.name}: n={w.n}, N={w.N}, keep_frac={args.keep_frac}, adaptive peer selection",
-                   "sample_columns": cols},
+        "config": workload_config(w, args.keep_frac, 1),
+        "sample_columns": cols,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def workload_config(w, keep_frac, world):
+    """The `config` object both arms print: what is computed per step, on which inputs."""
+    n, N = w.n, w.N
+    ld = (N + 31) // 32 * 32
+    in_bytes = 2 * 4 * n * N
+    resident = in_bytes < L2_BYTES
+    return {
+        "workload": f"{w.name}: n={n} workers, N={N} fp32 params each (per GPU), keep_frac={keep_frac}, "
+                    f"lr={w.lr}, adaptive peer selection on U[{w.bw_range[0]:g},{w.bw_range[1]:g}] Mb/s",
+        "step": "peer selection (Algorithm 3) + SGD step + round mask + wire-buffer pack + pair average",
+        "row_stride": ld,
+        "l2": (f"inputs are {in_bytes / 1e6:.1f} MB per step and fit in the 126 MB L2: an L2-resident run, "
+               f"no flush between steps, not an HBM figure") if resident else
+              (f"inputs are {in_bytes / 1e9:.2f} GB per step, far larger than the 126 MB L2: no flush needed"),
+        "sharding": "column shards, one per GPU, no collective" if world > 1 else "single GPU",
+    }
 
 
 # ------------------------------------------------------------------------------------------
@@ -277,24 +335,22 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {
-            "workload": f"{w.name}: n={n} workers, N={N} fp32 params each (per GPU), keep_frac={p}, "
-                        f"lr={w.lr}, adaptive peer selection on U[{w.bw_range[0]:g},{w.bw_range[1]:g}] Mb/s",
-            "step": "saps_select_peers + saps_round_pack (tile prefix-scan kernel + fused SGD/mask/emit/average kernel, which also counts the next round's mask per tile)",
-            "row_stride": ld, "l2": f"inputs are {2 * 4 * n * N / 1e9:.2f} GB per step, far larger than the 126 MB L2",
-            "sharding": "column shards, one per GPU, no collective" if world > 1 else "single GPU",
-        },
+        "config": dict(workload_config(w, p, world),
+                       gpu_step="saps_select_peers + saps_round_pack (tile prefix-scan kernel + fused "
+                                "SGD/mask/emit/average kernel, which also counts the next round's mask per tile)"),
         "effective_hbm_gbs": bytes_round * K / (elapsed_ms * 1e-3) / 1e9,
         "frac_of_8tbs": bytes_round * K / (elapsed_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
         "kept_columns": kept,
         "gpu_launches": 2 * K,
         "clocks": clocks,
         "roofline": {
-            "bound": "hbm", "kernel": "round_kernel<4,true,true> (fused SGD + mask + emit + pair average)",
+            "bound": "hbm" if 2 * 4 * n * N >= L2_BYTES else "l2-resident",
+            "kernel": "round_kernel<4,true,true> (fused SGD + mask + emit + pair average)",
             "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
             "frac": achieved / peak, "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
             "kernel_ms": k_ms, "algorithmic_bytes": bytes_round + bytes_emit,
-            "traffic": None if NCU_TRAFFIC_BYTES_PER_ELEMENT is None else NCU_TRAFFIC_BYTES_PER_ELEMENT * n * N,
+            "traffic": ncu_traffic(w.name, p),
+            "traffic_source": NCU_TRAFFIC["source"] if ncu_traffic(w.name, p) is not None else None,
         },
     }
 
@@ -340,12 +396,21 @@ def run_ours(args):
     }
     t += 30
 
+    # what was timed is also what is right: one more step of the same sequence, replayed by the
+    # CPU oracle on a few sampled rows (outside every timed region)
+    if rank == 0 and not args.no_verify:
+        result["verified"] = verify_step(sb, ctx, w, B, t, p, x, g, vals, idx, count, stream)
+    t += 1
+
+    if rank == 0 and world == 1 and not args.no_small_loop:
+        result["resnet20_scheduler_loop"] = measure_small_loop(sb, synth, stream, peak)
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = measure_cpu_baseline(args, w, x, g)
     if not args.no_e2e:
         e2e = measure_e2e(args, sb, sharding, w, ctx, B, t, x, g, world, col_offset, barrier)
         if rank == 0:
             result["e2e"] = e2e
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        result["cpu_baseline"] = measure_cpu_baseline(args, synth, w)
 
     sb.saps_destroy(ctx)
     if world > 1:
@@ -353,6 +418,85 @@ def run_ours(args):
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(result))
+        if "verified" in result and not result["verified"]["bit_identical"]:
+            raise SystemExit("bench.py: the GPU round differs from the CPU oracle on the sampled rows")
+
+
+def verify_step(sb, ctx, w, B, t, p, x, g, vals, idx, count, stream):
+    """Runs the next step of the timed sequence (same context, same call, so the per-tile counts
+    come from the previous kernel's run-ahead exactly as in the timed steps) and compares the
+    rows of two matched pairs, the count, the index list and those rows of the wire buffer with
+    the CPU oracle's round on the same inputs, bit for bit."""
+    import numpy as np
+    import torch
+
+    import oracle
+    n, N = w.n, w.N
+    pairs = sb.saps_select_peers(ctx, B, t, n)
+    rows = sorted({0, int(pairs[0]), n // 2 + 1, int(pairs[n // 2 + 1])})
+    local = {r: i for i, r in enumerate(rows)}
+    x_s = x[rows, :N].cpu().numpy()
+    g_s = g[rows, :N].cpu().numpy()
+    sb.saps_round_pack(ctx, x, g, w.lr, pairs, t, p, vals, idx, count, stream)
+    torch.cuda.synchronize()
+    status = sb.saps_status(ctx)
+    a = x_s.copy()
+    oracle.sgd(a, g_s, w.lr)
+    m = oracle.gossip_round(x_s, g_s, w.lr, [local[int(pairs[r])] for r in rows], w.seed, t, p)
+    kept = np.nonzero(m)[0].astype(np.uint32)
+    c = int(count.cpu().numpy().view(np.uint32)[0])
+    checks = {
+        "status_ok": status == 0,
+        "count": c == len(kept),
+        "idx": c == len(kept) and bool((idx[:c].cpu().numpy().view(np.uint32) == kept).all()),
+        "x_rows": bool((x[rows, :N].cpu().numpy().view(np.uint32) == x_s.view(np.uint32)).all()),
+        "wire_rows": c == len(kept) and bool((vals[rows, :c].cpu().numpy().view(np.uint32)
+                                              == a[:, kept].view(np.uint32)).all()),
+    }
+    return {"rows": rows, "round": t, "elements_compared": len(rows) * N, "kept_columns": c,
+            "checks": checks, "bit_identical": all(checks.values()),
+            "how": "one more saps_select_peers + saps_round_pack step of the timed sequence, replayed by the "
+                   "CPU oracle on the sampled rows from a snapshot taken just before it"}
+
+
+def measure_small_loop(sb, synth, stream, peak):
+    """The ResNet-20-sized configuration (L2-resident: a step is a 19 us kernel) through the
+    C-side scheduler loop saps_run_rounds_pack, T rounds per call, so that no Python call sits
+    between two rounds."""
+    import torch
+    w = synth.WORKLOADS["resnet20"]
+    n, N, p, T = w.n, w.N, w.keep_fracs[0], 100
+    ld = (N + 31) // 32 * 32
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(4242)
+    x = torch.empty(n, ld, dtype=torch.float32, device="cuda").normal_(0.0, w.x_std, generator=gen)
+    g = torch.empty(n, ld, dtype=torch.float32, device="cuda").normal_(0.0, w.g_std, generator=gen)
+    B = synth.bandwidth_matrix(n, *w.bw_range, seed=w.seed)
+    ctx = sb.saps_create_ld(n, N, ld, w.seed)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.empty(n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.empty(cap, dtype=torch.int32, device="cuda")
+    counts = torch.zeros(T, dtype=torch.int32, device="cuda")
+    t = 1
+    for _ in range(3):
+        sb.saps_run_rounds_pack(ctx, x, g, w.lr, t, T, p, vals, idx, counts, bandwidth=B, stream=stream)
+        t += T
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 5
+    e0.record(stream)
+    for _ in range(reps):
+        sb.saps_run_rounds_pack(ctx, x, g, w.lr, t, T, p, vals, idx, counts, bandwidth=B, stream=stream)
+        t += T
+    e1.record(stream)
+    torch.cuda.synchronize()
+    st = sb.saps_status(ctx)
+    sb.saps_destroy(ctx)
+    ms = e0.elapsed_time(e1) / (reps * T)
+    return {"value": 1e3 / ms, "unit": UNIT, "us_per_round": ms * 1e3, "rounds_per_call": T, "calls": reps,
+            "status": st, "effective_gbs_l2_resident": 12.0 * n * N / (ms * 1e-3) / 1e9,
+            "api": "saps_run_rounds_pack (peer selection + emitting round, 100 rounds per call)",
+            "note": "inputs (70 MB) stay in L2 between rounds: not an HBM figure"}
 
 
 def measure_e2e(args, sb, sharding, w, ctx, B, t, x_dev, g_dev, world, col_offset, barrier):
@@ -408,22 +552,68 @@ def measure_e2e(args, sb, sharding, w, ctx, B, t, x_dev, g_dev, world, col_offse
     resident = {"value": world * steps / rdt, "unit": UNIT, "ms_per_step": rdt / steps * 1e3,
                 "h2d_bytes_per_step": 4 * n * N, "d2h_bytes_per_step": 4 * n * cap + 4 * cap + 4,
                 "note": "model resident in HBM; gradients in from pinned host memory, wire buffer out"}
-    return {"value": world * steps / dt, "unit": UNIT, "model_resident": resident, "h2d_bytes_per_step": 2 * 4 * n * N,
-            "d2h_bytes_per_step": 4 * n * N + 4 * n * cap + 4 * cap + 4, "ms_per_step": dt / steps * 1e3,
-            "steps": steps, "kept_columns": int(hc.numpy().view("uint32")[0]),
-            "api": "saps_select_peers + saps_round_pack_host (pinned host x and g in; x, packed values, "
-                   "indices and count out; chunked copy/compute pipeline over 3 streams)"}
+    ms = dt / steps * 1e3
+    out = {"value": world * steps / dt, "unit": UNIT, "model_resident": resident, "h2d_bytes_per_step": 2 * 4 * n * N,
+           "d2h_bytes_per_step": 4 * n * N + 4 * n * cap + 4 * cap + 4, "ms_per_step": ms,
+           "steps": steps, "kept_columns": int(hc.numpy().view("uint32")[0]),
+           "api": "saps_select_peers + saps_round_pack_host (pinned host x and g in; x, packed values, "
+                  "indices and count out; column chunks copied in and computed on 3 streams, results "
+                  "copied out on a fourth)"}
+    if world == 1:
+        # what the link allows: the same bytes as bare pinned copies, nothing else running
+        bound = pcie_bound(torch, hx, hg, x_dev, g_dev, n, N)
+        out["pcie"] = dict(bound, frac_of_h2d_bound=bound["h2d_only_ms"] / ms,
+                           frac_of_bidirectional_bound=bound["bidirectional_ms"] / ms)
+    return out
 
 
-def measure_cpu_baseline(args, synth, w):
-    """The CPU oracle as it stands (one thread), on a bounded sample of the same workload."""
+def pcie_bound(torch, hx, hg, x_dev, g_dev, n, N):
+    """Time of bare pinned copies of one step's bytes: (a) the 2 x 4nN bytes host -> device alone,
+    (b) the same while 4nN bytes travel device -> host on another stream (what a perfectly
+    overlapped step would take).  The device buffers are used as flat scratch."""
+    flat_x, flat_g = x_dev.view(-1)[:n * N], g_dev.view(-1)[:n * N]
+    keep = flat_x.clone()
+    back = torch.empty(n * N, dtype=torch.float32).pin_memory()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+
+    def h2d():
+        with torch.cuda.stream(s_in):
+            flat_x.copy_(hx.view(-1), non_blocking=True)
+            flat_g.copy_(hg.view(-1), non_blocking=True)
+
+    best_in, best_both = float("inf"), float("inf")
+    for _ in range(3):
+        torch.cuda.synchronize()
+        e[0].record(s_in)
+        h2d()
+        e[1].record(s_in)
+        torch.cuda.synchronize()
+        best_in = min(best_in, e[0].elapsed_time(e[1]))
+        e[2].record(s_out)
+        e[0].record(s_in)
+        h2d()
+        e[1].record(s_in)
+        with torch.cuda.stream(s_out):
+            back.copy_(keep, non_blocking=True)
+        e[3].record(s_out)
+        torch.cuda.synchronize()
+        best_both = min(best_both, max(e[0].elapsed_time(e[1]), e[2].elapsed_time(e[3])))
+    return {"h2d_only_ms": best_in, "h2d_gbs": 2 * 4 * n * N / (best_in * 1e-3) / 1e9,
+            "bidirectional_ms": best_both}
+
+
+def measure_cpu_baseline(args, w, x_dev, g_dev):
+    """The CPU oracle as it stands (one thread) on the benchmark's own matrices, copied down from
+    the device: the whole model when it has at most ORACLE_MAX_COLUMNS columns."""
     import numpy as np
 
     import oracle
     from oracle import peer_selection as ps
-    cols = min(w.N, 1 << 22)
-    x = synth.gaussian_matrix(w.n, cols, w.x_std, w.seed, 0)
-    g = synth.gaussian_matrix(w.n, cols, w.g_std, w.seed, 1)
+    from paper_2002_09692_b200 import synth
+    cols, sample = oracle_sample(w)
+    x = np.ascontiguousarray(x_dev[:, :cols].cpu().numpy())
+    g = np.ascontiguousarray(g_dev[:, :cols].cpu().numpy())
     B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
     R = ps.new_timestamps(w.n)
     b_thres, t_thres = ps.default_b_thres(B), ps.default_t_thres(w.n)
@@ -434,9 +624,8 @@ def measure_cpu_baseline(args, synth, w):
         oracle_step(oracle, ps, x, g, w, B, R, 2 + r, args.keep_frac, b_thres, t_thres, cols)
     dt = (time.perf_counter() - t0) / rounds
     return {"value": (cols / w.N) / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "host_cores_present": os.cpu_count(),
-            "sample": f"{rounds} rounds over the first {cols} of {w.N} columns of all {w.n} workers; "
-                      f"rounds/s scaled by {cols}/{w.N}"}
+            "host_cores_present": os.cpu_count(), "ms_per_round": dt * 1e3,
+            "sample": f"{rounds} rounds (after 1 warm-up) over " + sample}
 
 
 def main():

@@ -131,7 +131,10 @@ SAPS_API int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, 
  * t (the mask does not depend on the data, and the integer units are idle in a memory-bound
  * kernel), so a following call for round t+1 with the same keep_frac only has to take a
  * prefix sum of a few thousand numbers.  Any other call counts in a kernel of its own.
- * Results are identical either way; enabled = 0 switches the run-ahead off. */
+ * Results are identical either way; enabled = 0 switches the run-ahead off.
+ * The counts are kept in the context and read by the next call's kernels, so consecutive
+ * emitting calls on one context must run on one stream or be ordered by events (the general
+ * rule above that calls on one context must not overlap covers it). */
 SAPS_API int saps_set_run_ahead(saps_ctx* ctx, int enabled);
 
 /* Order of the two halves of the update.
@@ -198,12 +201,13 @@ SAPS_API int saps_unpack_avg_rows(saps_ctx* ctx, float* x, const float* recv_val
  * process whose framework has already claimed the whole GPU for its own memory pool, a
  * latency-critical loop that cannot afford the device-wide synchronisation an allocation
  * implies, or a plug-in that is only handed buffers and a stream.  saps_pack would allocate
- * the context's scratch area on its first use; this variant never does.  It calls neither
- * cudaMalloc nor cudaFree nor any allocating library routine, now or later.
+ * the context's scratch area on its first use; this variant never does: it calls neither
+ * cudaMalloc nor cudaFree nor any library routine that does.
  *
  * Instead the tile states of the compaction scan live in a fixed array inside the library
- * image (786,448 bytes, present on every GPU that loads the library, until the process
- * exits).  That array covers N <= SAPS_NOALLOC_MAX_N columns; a larger context is refused
+ * image (786,448 bytes).  The CUDA runtime creates that array on a GPU when it loads the
+ * library's device code there (at the latest on the first launch of one of its kernels on
+ * that GPU), not on demand from this call, and keeps it until the process exits.  That array covers N <= SAPS_NOALLOC_MAX_N columns; a larger context is refused
  * with SAPS_ERR_TOO_LARGE before anything is launched.
  *
  * Arguments and results are those of saps_pack (same capacity rule, same overflow
@@ -239,7 +243,11 @@ SAPS_API int saps_set_select_params(saps_ctx* ctx, double b_thres, int t_thres);
  *              worker i could not be matched: odd n or missing links)
  * Records the chosen pairs in the context's timestamp matrix R.  t must not decrease
  * between calls (SAPS_ERR_INVALID).  Any maximum matching of the candidate edges is a
- * valid answer; which one is returned depends on (seed, t) only. */
+ * valid answer; which one is returned depends on (seed, t) only.
+ * Round numbers are kept as signed 64-bit timestamps: 1 <= t <= SAPS_SELECT_MAX_T, else
+ * SAPS_ERR_INVALID (the same limit holds for the rounds of saps_run_rounds* when they select
+ * peers, and for last_t and the entries of R given to saps_set_select_state). */
+#define SAPS_SELECT_MAX_T ((1ull << 62) - 1)
 SAPS_API int saps_select_peers(saps_ctx* ctx, const double* bandwidth, uint64_t t, int32_t* out_pairs);
 
 /* Forgets every recorded exchange (R = "never") and the last t. */
@@ -280,8 +288,10 @@ SAPS_API int saps_run_rounds_pack(saps_ctx* ctx, float* x, const float* g, float
 /* One round on HOST matrices: copies x_host and g_host ([n, N] fp32, row stride N; pinned
  * memory recommended) to the device staging buffers, runs the round, copies x back, all in
  * column chunks pipelined over internal streams, and waits for completion.
- *   d_x, d_g  device staging, n * ld_dev floats each, ld_dev = N rounded up to a multiple of
- *             32, 16-byte aligned; caller-owned.  g_host may be NULL (then lr = 0, d_g unused). */
+ *   d_x, d_g  device staging, [n, ld] fp32 with the context's row stride ld (create the
+ *             context with saps_create_ld and ld a multiple of 32 for 128-bit accesses);
+ *             caller-owned.  g_host may be NULL (then lr = 0, d_g unused).
+ * The first call creates the internal streams and events (not inside a stream capture). */
 SAPS_API int saps_round_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
                     const int32_t* pairs, uint64_t t, double keep_frac, float* d_x, float* d_g);
 
@@ -298,6 +308,12 @@ SAPS_API int saps_round_pack_host(saps_ctx* ctx, float* x_host, const float* g_h
                                   float* d_g, float* out_vals_host, uint32_t* out_idx_host,
                                   uint32_t* out_count_host, float* d_vals, uint32_t* d_idx,
                                   uint32_t* d_count);
+
+/* Tuning of the copy/compute pipeline behind the two host-buffer entry points: columns per
+ * chunk (rounded up to whole 2048-column tiles; default 1,048,576) and the number of streams
+ * that copy chunks in and run the round on them (1..6, default 3; results always leave on one
+ * further stream).  0 leaves a setting as it is.  Results do not depend on either. */
+SAPS_API int saps_set_host_pipeline(saps_ctx* ctx, uint64_t chunk_columns, int lanes);
 
 /* ---- consensus and communication metrics -------------------------------------------------------- */
 

@@ -25,6 +25,7 @@ SAPS_ERR_NOMEM = -6
 SAPS_ERR_TOO_LARGE = -7
 SAPS_NOALLOC_MAX_N = 134_217_728
 SAPS_NEVER = -(1 << 62)
+SAPS_SELECT_MAX_T = (1 << 62) - 1
 
 
 def _load() -> ctypes.CDLL:
@@ -70,6 +71,7 @@ _SIGNATURES = {
     "saps_debug_inject": (_i32, [_vp, _u32, _u32]),
     "saps_round_host": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp, _vp]),
     "saps_round_pack_host": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "saps_set_host_pipeline": (_i32, [_vp, _u64, _i32]),
     "saps_set_timing_events": (_i32, [_vp, _vp, _vp]),
     "saps_status": (_i32, [_vp, _vp, ctypes.POINTER(_i32)]),
     "saps_strerror": (ctypes.c_char_p, [_i32]),
@@ -295,6 +297,10 @@ def saps_round_pack_host(ctx, x_host, g_host, lr, pairs, t, keep_frac, d_x, d_g,
                                      _ptr(d_x), _ptr(d_g), _ptr(out_vals_host), _ptr(out_idx_host),
                                      _ptr(out_count_host), _ptr(d_vals), _ptr(d_idx), _ptr(d_count)),
            "saps_round_pack_host")
+
+
+def saps_set_host_pipeline(ctx, chunk_columns: int = 0, lanes: int = 0) -> None:
+    _check(_lib.saps_set_host_pipeline(ctx, chunk_columns, lanes), "saps_set_host_pipeline")
 
 
 def saps_set_timing_events(ctx, before, after) -> None:

@@ -314,8 +314,8 @@ __global__ void __launch_bounds__(kThreads) consensus_partial_kernel(const float
     }
     if constexpr (VEC == 4) {
         // the last (N mod 4) columns
-        const uint32_t k = nfull + tid;
-        if (k < N && col0 <= nfull && nfull < col0 + kTileCols) {
+        if ((uint32_t)tid < N - nfull && col0 <= nfull && nfull < col0 + kTileCols) {
+            const uint32_t k = nfull + tid;  // cannot wrap: tid < N - nfull
             const double pivot = (double)x[k];
             double sd = 0.0, sdd = 0.0;
             for (int i = 1; i < n; ++i) {

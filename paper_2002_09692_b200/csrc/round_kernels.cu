@@ -184,9 +184,10 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
                 }
             }
             if constexpr (VEC > 1) {
-                const uint32_t k = nfull + tid;  // the (N mod VEC) leftover columns belong to the last tile
-                if (k < a.N && col_tile <= nfull && nfull < col_tile + kTileCols)
-                    c += column_kept(a.col_offset + k, a.next_key) ? 1u : 0u;
+                // the (N mod VEC) leftover columns belong to the last tile; tid is compared with
+                // their number first, so that nfull + tid cannot wrap for N close to 2^32
+                if ((uint32_t)tid < a.N - nfull && col_tile <= nfull && nfull < col_tile + kTileCols)
+                    c += column_kept(a.col_offset + nfull + tid, a.next_key) ? 1u : 0u;
             }
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, d);

@@ -26,11 +26,16 @@ struct saps_ctx {
     // device scratch, allocated on first use on the then-current device
     void* scratch;
     int scratch_device;
-    // pipeline of the host-buffer entry point, created on first use
-    static constexpr int kLanes = 3;
-    cudaStream_t lane_stream[kLanes];
-    cudaEvent_t lane_event[kLanes];
+    // pipeline of the host-buffer entry point, created on first use: kMaxLanes streams that
+    // copy a column chunk in and run the round on it, one stream that copies results out
+    static constexpr int kMaxLanes = 6;
+    cudaStream_t lane_stream[kMaxLanes];
+    cudaEvent_t lane_event[kMaxLanes];
+    cudaStream_t out_stream;
+    cudaEvent_t scan_event;
     bool lanes_ready;
+    int host_lanes;             // lanes in use
+    uint32_t host_chunk_tiles;  // column tiles per chunk
     // Mask scan of the emitting round (saps_round_pack): kept columns per tile for the current
     // round and, counted ahead by the fused kernel itself, for the next one; their prefix.
     uint32_t* emit_mem;        // device: cnt[0][ntiles], cnt[1][ntiles], excl[ntiles]
@@ -95,7 +100,9 @@ RowGroups make_groups(int n, const int32_t* pairs, bool singles)
     return rg;
 }
 
-int ensure_scratch(saps_ctx* ctx)
+// The scratch is cleared on the stream of the call that creates it, so that the clear is
+// ordered before that call's kernels whatever kind of stream it is.
+int ensure_scratch(saps_ctx* ctx, cudaStream_t stream)
 {
     if (ctx->scratch != nullptr) return SAPS_OK;
     int dev = -1;
@@ -109,7 +116,7 @@ int ensure_scratch(saps_ctx* ctx)
         cudaGetLastError();
         return SAPS_ERR_NOMEM;
     }
-    if (cudaMemset(p, 0, bytes) != cudaSuccess) {
+    if (cudaMemsetAsync(p, 0, bytes, stream) != cudaSuccess) {
         cudaFree(p);
         cudaGetLastError();
         return SAPS_ERR_CUDA;
@@ -198,6 +205,8 @@ int saps_create_ld(int n, uint64_t N, uint64_t ld, uint64_t seed, saps_ctx** out
     ctx->scratch = nullptr;
     ctx->scratch_device = -1;
     ctx->lanes_ready = false;
+    ctx->host_lanes = 3;
+    ctx->host_chunk_tiles = 512;
     ctx->emit_mem = nullptr;
     ctx->emit_cur = 0;
     ctx->ahead_valid = false;
@@ -224,11 +233,14 @@ int saps_create(int n, uint64_t N, uint64_t seed, saps_ctx** out)
 int saps_destroy(saps_ctx* ctx)
 {
     if (ctx == nullptr) return SAPS_ERR_INVALID;
-    if (ctx->lanes_ready)
-        for (int l = 0; l < saps_ctx::kLanes; ++l) {
+    if (ctx->lanes_ready) {
+        for (int l = 0; l < saps_ctx::kMaxLanes; ++l) {
             cudaStreamDestroy(ctx->lane_stream[l]);
             cudaEventDestroy(ctx->lane_event[l]);
         }
+        cudaStreamDestroy(ctx->out_stream);
+        cudaEventDestroy(ctx->scan_event);
+    }
     if (ctx->scratch != nullptr) cudaFree(ctx->scratch);
     if (ctx->partials != nullptr) cudaFree(ctx->partials);
     if (ctx->emit_mem != nullptr) cudaFree(ctx->emit_mem);
@@ -412,7 +424,7 @@ int saps_pack(saps_ctx* ctx, const float* x, uint64_t t, double keep_frac, float
     if (ctx == nullptr || x == nullptr || out_vals == nullptr || out_count == nullptr || t == 0 ||
         !valid_frac(keep_frac))
         return SAPS_ERR_INVALID;
-    int rc = ensure_scratch(ctx);
+    int rc = ensure_scratch(ctx, (cudaStream_t)stream);
     if (rc != SAPS_OK) return rc;
     PackArgs a;
     a.x = x;
@@ -479,7 +491,7 @@ int ensure_emit_memory(saps_ctx* ctx)
 int prepare_emission(saps_ctx* ctx, uint64_t t, double keep_frac, uint32_t cap, uint32_t* out_idx,
                      uint32_t* out_count, float* out_vals, cudaStream_t stream, RoundArgs* a)
 {
-    int rc = ensure_scratch(ctx);
+    int rc = ensure_scratch(ctx, stream);
     if (rc != SAPS_OK) return rc;
     rc = ensure_emit_memory(ctx);
     if (rc != SAPS_OK) return rc;
@@ -556,7 +568,8 @@ int saps_set_select_params(saps_ctx* ctx, double b_thres, int t_thres)
 
 int saps_select_peers(saps_ctx* ctx, const double* bandwidth, uint64_t t, int32_t* out_pairs)
 {
-    if (ctx == nullptr || bandwidth == nullptr || out_pairs == nullptr || t == 0) return SAPS_ERR_INVALID;
+    if (ctx == nullptr || bandwidth == nullptr || out_pairs == nullptr || t == 0 || t > SAPS_SELECT_MAX_T)
+        return SAPS_ERR_INVALID;
     return select_peers(ctx->select, bandwidth, t, out_pairs);
 }
 
@@ -578,8 +591,12 @@ int saps_get_select_state(const saps_ctx* ctx, int64_t* out_R, uint64_t* out_las
 
 int saps_set_select_state(saps_ctx* ctx, const int64_t* R, uint64_t last_t)
 {
-    if (ctx == nullptr) return SAPS_ERR_INVALID;
-    if (R) std::memcpy(ctx->select.R.data(), R, ctx->select.R.size() * sizeof(int64_t));
+    if (ctx == nullptr || last_t > SAPS_SELECT_MAX_T) return SAPS_ERR_INVALID;
+    if (R) {
+        for (size_t e = 0; e < ctx->select.R.size(); ++e)
+            if (R[e] != kNever && (R[e] < 0 || (uint64_t)R[e] > SAPS_SELECT_MAX_T)) return SAPS_ERR_INVALID;
+        std::memcpy(ctx->select.R.data(), R, ctx->select.R.size() * sizeof(int64_t));
+    }
     ctx->select.last_t = last_t;
     return SAPS_OK;
 }
@@ -598,6 +615,7 @@ int run_rounds_impl(saps_ctx* ctx, float* x, const float* g, float lr, uint64_t 
     if (rc != SAPS_OK) return rc;
     if (pairs_list == nullptr && bandwidth == nullptr) return SAPS_ERR_INVALID;
     if (t_first + T < t_first) return SAPS_ERR_INVALID;
+    if (pairs_list == nullptr && T > 0 && t_first + T - 1 > SAPS_SELECT_MAX_T) return SAPS_ERR_INVALID;
     if (lr_list != nullptr) {
         if (g == nullptr) return SAPS_ERR_INVALID;
         for (uint64_t r = 0; r < T; ++r)
@@ -671,27 +689,36 @@ struct HostPack {
 int ensure_lanes(saps_ctx* ctx)
 {
     if (ctx->lanes_ready) return SAPS_OK;
+    constexpr int kStreams = saps_ctx::kMaxLanes + 1, kEvents = saps_ctx::kMaxLanes + 1;
+    cudaStream_t streams[kStreams];
+    cudaEvent_t events[kEvents];
     int ns = 0, ne = 0;
-    while (ns < saps_ctx::kLanes &&
-           cudaStreamCreateWithFlags(&ctx->lane_stream[ns], cudaStreamNonBlocking) == cudaSuccess)
-        ++ns;
-    while (ns == saps_ctx::kLanes && ne < saps_ctx::kLanes &&
-           cudaEventCreateWithFlags(&ctx->lane_event[ne], cudaEventDisableTiming) == cudaSuccess)
+    while (ns < kStreams && cudaStreamCreateWithFlags(&streams[ns], cudaStreamNonBlocking) == cudaSuccess) ++ns;
+    while (ns == kStreams && ne < kEvents &&
+           cudaEventCreateWithFlags(&events[ne], cudaEventDisableTiming) == cudaSuccess)
         ++ne;
-    if (ne != saps_ctx::kLanes) {
-        for (int m = 0; m < ne; ++m) cudaEventDestroy(ctx->lane_event[m]);
-        for (int m = 0; m < ns; ++m) cudaStreamDestroy(ctx->lane_stream[m]);
+    if (ne != kEvents) {
+        for (int m = 0; m < ne; ++m) cudaEventDestroy(events[m]);
+        for (int m = 0; m < ns; ++m) cudaStreamDestroy(streams[m]);
         cudaGetLastError();
         return SAPS_ERR_CUDA;
     }
+    for (int l = 0; l < saps_ctx::kMaxLanes; ++l) {
+        ctx->lane_stream[l] = streams[l];
+        ctx->lane_event[l] = events[l];
+    }
+    ctx->out_stream = streams[saps_ctx::kMaxLanes];
+    ctx->scan_event = events[saps_ctx::kMaxLanes];
     ctx->lanes_ready = true;
     return SAPS_OK;
 }
 
-// The round acts column by column, so column chunks are independent: copy in, compute and
-// copy out chunk by chunk, round-robin over a few streams, so that the two copy directions
-// and the kernels overlap.  With a wire buffer, the mask scan (which touches no model data)
-// runs first on lane 0 and the other lanes wait for its tile prefixes.
+// The round acts column by column, so column chunks are independent.  Each chunk is copied in
+// and computed on one of a few lane streams (round-robin); its result is copied out on a
+// stream of its own, so that a lane can start its next copy-in without waiting for its last
+// copy-out: the two copy directions and the kernels overlap, and the copy-in queue never
+// runs dry.  With a wire buffer, the mask scan (which touches no model data) runs first on
+// lane 0 and the other lanes wait for its tile prefixes.
 int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr, const int32_t* pairs,
                     uint64_t t, double keep_frac, float* d_x, float* d_g, const HostPack* pack)
 {
@@ -707,8 +734,9 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
     rc = ensure_lanes(ctx);
     if (rc != SAPS_OK) return rc;
     const int n = ctx->n;
+    const int lanes = ctx->host_lanes;
     const uint64_t N = ctx->N;
-    const uint64_t ld_dev = (N + 31) / 32 * 32;
+    const uint64_t ld_dev = ctx->ld;   // the staging matrices use the context's row stride
     const bool emit = pack != nullptr;
     const RowGroups rg = make_groups(n, pairs, g_host != nullptr || emit);
     const RoundKey key = make_key(ctx->seed, t, keep_frac);
@@ -720,13 +748,13 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
         rc = prepare_emission(ctx, t, keep_frac, cap, pack->idx_host != nullptr ? pack->d_idx : nullptr,
                               pack->d_count, pack->d_vals, ctx->lane_stream[0], &emit_args);
         if (rc != SAPS_OK) return rc;
-        failed |= cudaEventRecord(ctx->lane_event[0], ctx->lane_stream[0]) != cudaSuccess;
-        for (int l = 1; l < saps_ctx::kLanes; ++l)
-            failed |= cudaStreamWaitEvent(ctx->lane_stream[l], ctx->lane_event[0], 0) != cudaSuccess;
+        failed |= cudaEventRecord(ctx->scan_event, ctx->lane_stream[0]) != cudaSuccess;
+        for (int l = 1; l < lanes; ++l)
+            failed |= cudaStreamWaitEvent(ctx->lane_stream[l], ctx->scan_event, 0) != cudaSuccess;
     }
-    const uint32_t tiles_per_chunk = 512;  // 1 Mi columns: n x 4 MiB per matrix and chunk
+    const uint32_t tiles_per_chunk = ctx->host_chunk_tiles;
     int lane = 0;
-    for (uint32_t tb = 0; tb < ctx->ntiles && !failed; tb += tiles_per_chunk, lane = (lane + 1) % saps_ctx::kLanes) {
+    for (uint32_t tb = 0; tb < ctx->ntiles && !failed; tb += tiles_per_chunk, lane = (lane + 1) % lanes) {
         const uint32_t tc = ctx->ntiles - tb < tiles_per_chunk ? ctx->ntiles - tb : tiles_per_chunk;
         const uint64_t c0 = (uint64_t)tb * kTileCols;
         const uint64_t c1 = c0 + (uint64_t)tc * kTileCols < N ? c0 + (uint64_t)tc * kTileCols : N;
@@ -742,26 +770,26 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
         a.tile_begin = tb;
         a.tile_count = tc;
         failed |= launch_round(a, emit, s) != cudaSuccess;
+        // everything that leaves the device does so on out_stream, behind this chunk's kernel
+        failed |= cudaEventRecord(ctx->lane_event[lane], s) != cudaSuccess;
+        failed |= cudaStreamWaitEvent(ctx->out_stream, ctx->lane_event[lane], 0) != cudaSuccess;
         if (x_host != nullptr)
             failed |= cudaMemcpy2DAsync(x_host + c0, N * sizeof(float), d_x + c0, ld_dev * sizeof(float), width, n,
-                                        cudaMemcpyDeviceToHost, s) != cudaSuccess;
+                                        cudaMemcpyDeviceToHost, ctx->out_stream) != cudaSuccess;
     }
     if (emit && !failed) {
-        // the wire buffer is complete once every lane has run its chunks
-        cudaStream_t s0 = ctx->lane_stream[0];
-        for (int l = 1; l < saps_ctx::kLanes; ++l) {
-            failed |= cudaEventRecord(ctx->lane_event[l], ctx->lane_stream[l]) != cudaSuccess;
-            failed |= cudaStreamWaitEvent(s0, ctx->lane_event[l], 0) != cudaSuccess;
-        }
-        failed |= cudaMemcpyAsync(pack->count_host, pack->d_count, sizeof(uint32_t), cudaMemcpyDeviceToHost, s0) !=
+        // out_stream has waited for every chunk's kernel, so the wire buffer is complete there
+        cudaStream_t so = ctx->out_stream;
+        failed |= cudaMemcpyAsync(pack->count_host, pack->d_count, sizeof(uint32_t), cudaMemcpyDeviceToHost, so) !=
                   cudaSuccess;
         failed |= cudaMemcpyAsync(pack->vals_host, pack->d_vals, (size_t)n * cap * sizeof(float),
-                                  cudaMemcpyDeviceToHost, s0) != cudaSuccess;
+                                  cudaMemcpyDeviceToHost, so) != cudaSuccess;
         if (pack->idx_host != nullptr)
             failed |= cudaMemcpyAsync(pack->idx_host, pack->d_idx, (size_t)cap * sizeof(uint32_t),
-                                      cudaMemcpyDeviceToHost, s0) != cudaSuccess;
+                                      cudaMemcpyDeviceToHost, so) != cudaSuccess;
     }
-    for (int l = 0; l < saps_ctx::kLanes; ++l) failed |= cudaStreamSynchronize(ctx->lane_stream[l]) != cudaSuccess;
+    for (int l = 0; l < lanes; ++l) failed |= cudaStreamSynchronize(ctx->lane_stream[l]) != cudaSuccess;
+    failed |= cudaStreamSynchronize(ctx->out_stream) != cudaSuccess;
     if (failed) {
         ctx->ahead_valid = false;
         cudaGetLastError();
@@ -771,6 +799,17 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
 }
 
 }  // namespace
+
+int saps_set_host_pipeline(saps_ctx* ctx, uint64_t chunk_columns, int lanes)
+{
+    if (ctx == nullptr || lanes < 0 || lanes > saps_ctx::kMaxLanes) return SAPS_ERR_INVALID;
+    if (chunk_columns != 0) {
+        const uint64_t tiles = (chunk_columns + kTileCols - 1) / kTileCols;
+        ctx->host_chunk_tiles = tiles > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)tiles;
+    }
+    if (lanes != 0) ctx->host_lanes = lanes;
+    return SAPS_OK;
+}
 
 int saps_round_host(saps_ctx* ctx, float* x_host, const float* g_host, float lr, const int32_t* pairs,
                     uint64_t t, double keep_frac, float* d_x, float* d_g)
@@ -796,9 +835,14 @@ int saps_status(saps_ctx* ctx, void* stream, int* out_device_status)
     }
     *out_device_status = SAPS_OK;
     if (ctx->scratch == nullptr) return SAPS_OK;
+    // read and clear on the caller's stream: a non-blocking stream is not ordered with the
+    // legacy default stream, and the clear must not land behind a later kernel's report
+    cudaStream_t s = (cudaStream_t)stream;
     int st = 0;
-    if (cudaMemcpy(&st, ctx->scratch, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess ||
-        (st != 0 && cudaMemset(ctx->scratch, 0, sizeof(int)) != cudaSuccess)) {
+    if (cudaMemcpyAsync(&st, ctx->scratch, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess ||
+        (st != 0 && (cudaMemsetAsync(ctx->scratch, 0, sizeof(int), s) != cudaSuccess ||
+                     cudaStreamSynchronize(s) != cudaSuccess))) {
         cudaGetLastError();
         return SAPS_ERR_CUDA;
     }

@@ -96,6 +96,37 @@ def test_round_rejects_bad_arguments_before_any_launch():
     assert sb.saps_strerror(-99) == "unknown status"
 
 
+def test_selection_round_numbers_stay_inside_the_signed_timestamp_range():
+    # round numbers become signed 64-bit timestamps in R; anything that could wrap, or collide
+    # with the "never" marker, is refused on the host
+    n = 4
+    B = np.ones((n, n)) - np.eye(n)
+    ctx = sb.saps_create(n, 100, 0)
+    out = (ctypes.c_int32 * n)()
+    big = sb.SAPS_SELECT_MAX_T
+    assert sb._lib.saps_select_peers(ctx, B.ctypes.data, big + 1, out) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_select_peers(ctx, B.ctypes.data, 1 << 63, out) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_select_peers(ctx, B.ctypes.data, (1 << 64) - 1, out) == sb.SAPS_ERR_INVALID
+    assert sb.saps_get_select_state(ctx, n)[1] == 0                       # nothing was recorded
+    fake = 0x1000
+    # the scheduler refuses before it launches anything when a later round would cross the limit
+    assert sb._lib.saps_run_rounds(ctx, fake, fake, 0.1, big, 2, 0.5, None, None, B.ctypes.data, None,
+                                   None) == sb.SAPS_ERR_INVALID
+    R_ok = (ctypes.c_int64 * (n * n))(*([sb.SAPS_NEVER] * (n * n)))
+    assert sb._lib.saps_set_select_state(ctx, R_ok, big + 1) == sb.SAPS_ERR_INVALID
+    for bad in (-1, big + 1, -(1 << 63)):
+        R_bad = (ctypes.c_int64 * (n * n))(*([sb.SAPS_NEVER] * (n * n)))
+        R_bad[1] = bad
+        assert sb._lib.saps_set_select_state(ctx, R_bad, 5) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_set_select_state(ctx, R_ok, big - 1) == sb.SAPS_OK
+    # the largest allowed round still works and is recorded as it is
+    pairs = sb.saps_select_peers(ctx, B, big, n)
+    check_involution(pairs)
+    R, last = sb.saps_get_select_state(ctx, n)
+    assert last == big and R[0][pairs[0]] == big
+    sb.saps_destroy(ctx)
+
+
 def test_pack_capacity_formula():
     ctx = sb.saps_create(32, 14_728_266, 0)
     for p in (0.1, 0.01, 0.001):

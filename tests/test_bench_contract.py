@@ -35,3 +35,35 @@ def test_reference_arm_prints_one_json_line():
 
 def test_reference_arm_other_ranks_print_nothing():
     assert _run({"RANK": "1", "WORLD_SIZE": "2", "LOCAL_RANK": "1"}, "--steps", "1", "--warmup", "1") == ""
+
+
+def test_reference_arm_runs_the_whole_default_workload():
+    # the default workload is timed at full width by the oracle (no scaling), larger ones on a
+    # stated column sample
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2002_09692_b200 import synth
+    cols, sample = bench.oracle_sample(synth.WORKLOADS["vgg16"])
+    assert cols == synth.WORKLOADS["vgg16"].N and "nothing scaled" in sample
+    cols, sample = bench.oracle_sample(synth.WORKLOADS["gpt2s"])
+    assert cols == bench.ORACLE_MAX_COLUMNS < synth.WORKLOADS["gpt2s"].N and "scaled by" in sample
+    small = bench.workload_config(synth.WORKLOADS["resnet20"], 0.01, 1)
+    assert "L2-resident" in small["l2"]
+    big = bench.workload_config(synth.WORKLOADS["vgg16"], 0.01, 1)
+    assert "far larger" in big["l2"]
+
+
+def test_recorded_dram_traffic_is_tied_to_the_kernel_sources():
+    # the ncu figure is reported only for the workload it was captured on and only while the
+    # kernel's sources are the ones that were captured
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.ncu_traffic("resnet20", 0.01) is None
+    assert bench.ncu_traffic("vgg16", 0.001) is None
+    got = bench.ncu_traffic("vgg16", 0.01)
+    if bench.NCU_TRAFFIC["kernel_sources_sha256"] == bench.kernel_sources_hash():
+        assert got == bench.NCU_TRAFFIC["bytes_per_launch"]
+        algorithmic = 12 * 32 * 14_728_266
+        assert 0.9 * algorithmic < got < 1.1 * algorithmic
+    else:
+        assert got is None

@@ -32,109 +32,184 @@ def _golden_count(seed, t, N, p):
     return None
 
 
-def test_vgg16_two_whole_rounds(sb):
+def _oracle_round_with_pack(x, g, w, pairs, t, p, cap):
+    """One round of the oracle in Algorithm 2's order, in place on x; returns the wire buffer."""
+    oracle.sgd(x, g, w.lr)
+    m = oracle.mask(w.seed, t, p, w.N)
+    wv, wi, wc = oracle.pack(x, m, cap)
+    oracle.pair_average(x, np.asarray(pairs, dtype=np.int32), m)
+    return wv, wi, wc
+
+
+def test_vgg16_consecutive_rounds_every_element(sb):
+    # The mode the benchmark times, at the size it times it: one context, keep_frac fixed at
+    # 0.01, saps_select_peers + saps_round_pack on consecutive rounds, so that from the second
+    # round on the per-tile counts (7,192 tiles) are the ones the previous fused kernel counted
+    # ahead.  Every element of x, the count, the index list and the packed values are compared
+    # with the oracle after every round.  A fourth round at keep_frac 0.001 then takes the
+    # other route (counts from a kernel of their own).  The same first three rounds are then
+    # repeated from the initial model through the C-side loop saps_run_rounds_pack.
     torch = torch_cuda()
     w = synth.WORKLOADS["vgg16"]
     n, N, ld = w.n, w.N, round_up(w.N, 32)
     x, g = synth.model_and_grad(w)
+    x0 = x.copy()
     B = synth.bandwidth_matrix(n, *w.bw_range, seed=w.seed)
     dx = torch.zeros(n, ld, dtype=torch.float32, device="cuda")
     dg = torch.zeros(n, ld, dtype=torch.float32, device="cuda")
     dx[:, :N].copy_(torch.from_numpy(x))
     dg[:, :N].copy_(torch.from_numpy(g))
     ctx = sb.saps_create_ld(n, N, ld, w.seed)
-    for p in w.keep_fracs:                               # 0.01, then 0.001
+    schedule = [(1, 0.01), (2, 0.01), (3, 0.01), (4, 0.001)]
+    used_pairs, counts3 = [], []
+    last3 = None
+    for t, p in schedule:
         cap = sb.saps_pack_capacity(ctx, p)
         vals = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
         idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
         count = torch.zeros(1, dtype=torch.int32, device="cuda")
-        t = 1 if p == 0.01 else 2
         pairs = sb.saps_select_peers(ctx, B, t, n)
         sb.saps_round_pack(ctx, dx, dg, w.lr, pairs, t, p, vals, idx, count)
         torch.cuda.synchronize()
         assert sb.saps_status(ctx) == 0
-        oracle.sgd(x, g, w.lr)
-        m = oracle.mask(w.seed, t, p, N)
-        wv, wi, wc = oracle.pack(x, m, cap)
-        oracle.pair_average(x, pairs, m)
-        if t == 1:
+        wv, wi, wc = _oracle_round_with_pack(x, g, w, pairs, t, p, cap)
+        if (t, p) == (1, 0.01):
             assert wc == _golden_count(0, 1, N, p) == 147_227
-        assert int(count[0]) == wc
-        assert (idx[:wc].cpu().numpy().view(np.uint32) == wi[:wc]).all()
-        assert_bits_equal(vals[:, :wc].cpu().numpy(), wv[:, :wc], f"wire buffer, keep_frac {p}")
+        assert int(count[0]) == wc, f"count of round {t}"
+        assert (idx[:wc].cpu().numpy().view(np.uint32) == wi[:wc]).all(), f"index list of round {t}"
+        assert_bits_equal(vals[:, :wc].cpu().numpy(), wv[:, :wc], f"wire buffer of round {t}")
         assert_bits_equal(dx[:, :N].cpu().numpy(), x, f"model after round {t}")
         assert float(dx[:, N:].abs().max()) == 0.0       # padding columns untouched
+        if p == 0.01:
+            used_pairs.append(pairs)
+            counts3.append(wc)
+            if t == 3:
+                last3 = (x.copy(), wv[:, :wc].copy(), wi[:wc].copy())
     sb.saps_destroy(ctx)
+    del x
+
+    # the same three rounds through the scheduler loop, selection included, in one call
+    want_x, want_v, want_i = last3
+    dx[:, :N].copy_(torch.from_numpy(x0))
+    ctx = sb.saps_create_ld(n, N, ld, w.seed)
+    cap = sb.saps_pack_capacity(ctx, 0.01)
+    vals = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    counts = torch.zeros(3, dtype=torch.int32, device="cuda")
+    log = np.zeros((3, n), dtype=np.int32)
+    sb.saps_run_rounds_pack(ctx, dx, dg, w.lr, 1, 3, 0.01, vals, idx, counts, bandwidth=B, out_pairs_log=log)
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    sb.saps_destroy(ctx)
+    assert log.tolist() == [list(p) for p in used_pairs]          # same matchings as call by call
+    assert counts.cpu().numpy().view(np.uint32).tolist() == counts3
+    c = counts3[-1]
+    assert (idx[:c].cpu().numpy().view(np.uint32) == want_i).all()
+    assert_bits_equal(vals[:, :c].cpu().numpy(), want_v, "wire buffer of round 3 from the scheduler loop")
+    assert_bits_equal(dx[:, :N].cpu().numpy(), want_x, "model after three scheduled rounds")
+    assert float(dx[:, N:].abs().max()) == 0.0
 
 
-def _sampled_round(sb, torch, w, p, t, pairs, sample_rows, golden=None):
-    """One bench-style round on device-drawn inputs; returns nothing, asserts parity."""
+def _sampled_rounds(sb, torch, w, p, pairs_of_round, rows_of_round, golden=None):
+    """Bench-style consecutive rounds t = 1, 2, ... on one context (fixed keep_frac, so every
+    round after the first uses the counts the previous kernel took ahead) on device-drawn
+    inputs.  After every round: the sampled rows against the oracle element by element, the
+    index list and the count against the oracle's mask, and properties that hold at any size
+    on all rows with device arithmetic.  rows_of_round[t-1] is closed under round t's matching
+    and contains rows_of_round[t]: the oracle follows exactly the rows whose whole history it
+    has seen."""
     n, N, ld = w.n, w.N, round_up(w.N, 32)
     gen = torch.Generator(device="cuda")
-    gen.manual_seed(99 + t)
+    gen.manual_seed(99 + int(p * 1e6))
     dx = torch.empty(n, ld, dtype=torch.float32, device="cuda").normal_(0.0, w.x_std, generator=gen)
     dg = torch.empty(n, ld, dtype=torch.float32, device="cuda").normal_(0.0, w.g_std, generator=gen)
-    rows = sorted(sample_rows)
-    x_s = dx[rows, :N].cpu().numpy()
-    g_s = dg[rows, :N].cpu().numpy()
-    a_dev = dx - w.lr * dg                              # two roundings per element, like the round
+    first = sorted(rows_of_round[0])
+    state = {r: dx[r, :N].cpu().numpy() for r in first}              # the oracle's copy of the rows
+    grad = {r: dg[r, :N].cpu().numpy() for r in first}
     ctx = sb.saps_create_ld(n, N, ld, w.seed)
     cap = sb.saps_pack_capacity(ctx, p)
     vals = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
     idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
     count = torch.zeros(1, dtype=torch.int32, device="cuda")
     bits = torch.zeros(round_up(N, 32) // 32, dtype=torch.int32, device="cuda")
-    sb.saps_mask(ctx, t, p, bits)
-    sb.saps_round_pack(ctx, dx, dg, w.lr, pairs, t, p, vals, idx, count)
-    torch.cuda.synchronize()
-    assert sb.saps_status(ctx) == 0
+    shifts = torch.arange(32, device="cuda", dtype=torch.int32)
+    for t, pairs in enumerate(pairs_of_round, start=1):
+        rows = sorted(rows_of_round[t - 1])
+        local = {r: i for i, r in enumerate(rows)}
+        assert all(int(pairs[r]) in local for r in rows) and all(r in state for r in rows)
+        a = (dx - w.lr * dg)[:, :N]                       # two roundings per element, like the round
+        sb.saps_mask(ctx, t, p, bits)
+        sb.saps_round_pack(ctx, dx, dg, w.lr, pairs, t, p, vals, idx, count)
+        torch.cuda.synchronize()
+        assert sb.saps_status(ctx) == 0
+
+        # -- element by element on the sampled rows --
+        x_s = np.stack([state[r] for r in rows])
+        g_s = np.stack([grad[r] for r in rows])
+        m = oracle.gossip_round(x_s, g_s, w.lr, [local[int(pairs[r])] for r in rows], w.seed, t, p)
+        for i, r in enumerate(rows):
+            state[r] = x_s[i]
+        c = int(count[0])
+        assert c == int(m.sum(dtype=np.int64)), f"count of round {t}"
+        if golden is not None and t == 1:
+            assert c == golden
+        assert_bits_equal(dx[rows, :N].cpu().numpy(), x_s, f"sampled rows {rows}, round {t}")
+        kept = np.nonzero(m)[0]
+        assert (idx[:c].cpu().numpy().view(np.uint32) == kept.astype(np.uint32)).all(), f"index list, round {t}"
+        del x_s, g_s
+
+        # -- properties on every row, on the device --
+        mdev = ((bits[:, None] >> shifts[None, :]) & 1).bool().reshape(-1)[:N]
+        assert int(mdev.sum()) == c
+        out = dx[:, :N]
+        peer = torch.as_tensor(np.asarray(pairs), device="cuda", dtype=torch.long)
+        assert torch.equal(torch.where(mdev[None, :], a, out), a)               # unmasked: SGD step only
+        om, am = out[:, mdev], a[:, mdev]
+        assert torch.equal(om, om[peer])                                        # peers agree bitwise
+        assert torch.equal(om + om[peer], am + am[peer])                        # pair sums to one rounding
+        assert torch.equal(vals[:, :c], am)                                     # wire buffer = a o m
+        del a, mdev, out, om, am
     sb.saps_destroy(ctx)
 
-    # -- element by element on the sampled rows --
-    local = {r: i for i, r in enumerate(rows)}
-    sub_pairs = [local[int(pairs[r])] for r in rows]
-    m = oracle.gossip_round(x_s, g_s, w.lr, sub_pairs, w.seed, t, p)
-    c = int(count[0])
-    assert c == int(m.sum(dtype=np.int64))
-    if golden is not None:
-        assert c == golden
-    assert_bits_equal(dx[rows, :N].cpu().numpy(), x_s, f"sampled rows {rows}")
-    kept = np.nonzero(m)[0]
-    assert (idx[:c].cpu().numpy().view(np.uint32) == kept.astype(np.uint32)).all()
 
-    # -- properties on every row, on the device --
-    shifts = torch.arange(32, device="cuda", dtype=torch.int32)
-    mdev = ((bits[:, None] >> shifts[None, :]) & 1).bool().reshape(-1)[:N]
-    assert int(mdev.sum()) == c
-    out = dx[:, :N]
-    a = a_dev[:, :N]
-    peer = torch.as_tensor(np.asarray(pairs), device="cuda", dtype=torch.long)
-    assert torch.equal(torch.where(mdev[None, :], a, out), a)                  # unmasked: SGD step only
-    assert torch.equal(out[:, mdev], out[peer][:, mdev])                        # peers agree bitwise
-    assert torch.equal(out[:, mdev] + out[peer][:, mdev], a[:, mdev] + a[peer][:, mdev])  # pair sums
-    assert torch.equal(vals[:, :c], a[:, mdev])                                 # wire buffer = a o m
+def _history_cone(pairs_of_round, last_rows):
+    """rows[t]: the workers whose values influence `last_rows` from round t+1 on, i.e. the set to
+    follow in round t+1: rows[T-1] = last_rows + their peers in round T, rows[t-1] = rows[t] +
+    their peers in round t."""
+    rows = [None] * len(pairs_of_round)
+    cur = set(last_rows)
+    for t in range(len(pairs_of_round) - 1, -1, -1):
+        cur = cur | {int(pairs_of_round[t][r]) for r in cur}
+        rows[t] = set(cur)
+    return rows
 
 
 def test_resnet50_keep_frac_sweep_sampled_rows(sb):
+    # uniformly random perfect matchings; three consecutive rounds per keep_frac on one context;
+    # the oracle follows workers 0 and 17 and everyone whose values reach them (at most 16 rows
+    # in round 1, 8 in round 2, 4 in round 3)
     torch = torch_cuda()
     w = synth.WORKLOADS["resnet50"]
     rng = synth.matching_rng(w.seed)
     for p in w.keep_fracs:
-        pairs = synth.random_perfect_matching(w.n, rng)
-        rows = {0, int(pairs[0]), 17, int(pairs[17])}
-        _sampled_round(sb, torch, w, p, 1, pairs, rows, golden=_golden_count(2, 1, w.N, p))
+        rounds = [synth.random_perfect_matching(w.n, rng) for _ in range(3)]
+        _sampled_rounds(sb, torch, w, p, rounds, _history_cone(rounds, {0, 17}),
+                        golden=_golden_count(2, 1, w.N, p))
         torch.cuda.empty_cache()
 
 
 def test_gpt2s_sampled_rows(sb):
+    # adaptive peer selection (Algorithm 3) for three consecutive rounds; the oracle follows
+    # worker 5 and everyone whose values reach it (8 rows in round 1, 4 in round 2, 2 in round 3)
     torch = torch_cuda()
     w = synth.WORKLOADS["gpt2s"]
     B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
     ctx = sb.saps_create(w.n, 16, w.seed)
-    pairs = sb.saps_select_peers(ctx, B, 1, w.n)
+    rounds = [sb.saps_select_peers(ctx, B, t, w.n) for t in (1, 2, 3)]
     sb.saps_destroy(ctx)
-    rows = {5, int(pairs[5])}
-    _sampled_round(sb, torch, w, 0.01, 1, pairs, rows, golden=_golden_count(0, 1, w.N, 0.01))
+    rows = _history_cone(rounds, {5})
+    assert len(rows[0]) <= 8 and len(rows[2]) == 2
+    _sampled_rounds(sb, torch, w, 0.01, rounds, rows, golden=_golden_count(0, 1, w.N, 0.01))
     torch.cuda.empty_cache()
 
 
@@ -195,6 +270,47 @@ def test_largest_column_count(sb):
     assert sb.saps_status(ctx) == 0
     assert int(count2.cpu().numpy().view(np.uint32)[0]) == c and torch.equal(idx2[:c], idx[:c])
     assert torch.equal(vals2[:, :c], x[:, gather])
+    del vals, idx, vals2, idx2, gather, mean, x0
+    torch.cuda.empty_cache()
+    # Two more rounds at a dense keep_frac: the second one takes its per-tile counts from the
+    # first one's kernel, which counted them ahead; with N mod 4 = 3 the three leftover columns
+    # are counted one thread each, and nfull + thread index must not wrap past 2^32 (a wrap
+    # would count columns 0..247 a second time: 12 spurious hits expected at this density).
+    p2 = 0.05
+    cap2 = sb.saps_pack_capacity(ctx, p2)
+    vals = torch.zeros(n, cap2, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap2, dtype=torch.int32, device="cuda")
+    for t2 in (t + 1, t + 2):
+        sb.saps_round_pack(ctx, x, None, 0.0, [1, 0], t2, p2, vals, idx, count)
+        sb.saps_mask(ctx, t2, p2, bits)
+        torch.cuda.synchronize()
+        assert sb.saps_status(ctx) == 0
+        c2 = int(count.cpu().numpy().view(np.uint32)[0])
+        words = bits.cpu().numpy().view(np.uint32)
+        assert c2 == int(np.bitwise_count(words).sum(dtype=np.int64)), f"count of round {t2}"
+        cols = idx[:c2].cpu().numpy().view(np.uint32)
+        assert int(cols[-1]) < N and int(cols[0]) >= 0
+        lo = N - 2 ** 12
+        k0, k1 = oracle.round_key(seed, t2)
+        thr2 = oracle.threshold(p2)
+        assert [int(k) for k in cols[cols >= lo]] == [k for k in range(lo, N) if oracle.hash_k(k, k0, k1) < thr2]
+    del vals, idx
+    torch.cuda.empty_cache()
+    # consensus distance at this size: both workers identical (the keep_frac = 1 round makes them
+    # so) except for one column that differs by exactly 1: || X - mean ||_F^2 = 2 * (1/2)^2
+    sb.saps_round(ctx, x, None, 0.0, [1, 0], t + 3, 1.0)
+    x[0, 0] = 0.25
+    x[1, 0] = 1.25
+    out = torch.zeros(1, dtype=torch.float64, device="cuda")
+    sb.saps_consensus_distance(ctx, x, out)
+    torch.cuda.synchronize()
+    assert float(out[0]) == 0.5
+    x[1, 0] = 0.25
+    x[0, N - 1] = 0.5                                    # the very last column, served by the leftover path
+    x[1, N - 1] = 2.5
+    sb.saps_consensus_distance(ctx, x, out)
+    torch.cuda.synchronize()
+    assert float(out[0]) == 2.0                          # 2 * (2/2)^2
     sb.saps_destroy(ctx)
-    del x, x0
+    del x
     torch.cuda.empty_cache()

@@ -259,3 +259,67 @@ def test_threshold_comparison_is_strict_on_the_gpu(sb):
             word = int(bits[k >> 5].cpu().numpy().view(np.uint32))
             assert (word >> (k & 31)) & 1 == want
     sb.saps_destroy(ctx)
+
+
+@pytest.mark.parametrize("N,ld", [(70_003, 70_016), (70_003, 70_003), (70_002, 70_002)])   # 128-, 32-, 64-bit access
+@pytest.mark.parametrize("scheduler", [False, True])
+def test_fused_emission_overflow_is_clamped_and_reported(sb, N, ld, scheduler):
+    # The count is Binomial(N, p), so a hard wire-buffer size can be exceeded (Eq. 2 / Section II-B).
+    # With a capacity below the true count the emitting round must: keep the model exactly
+    # right, report the true count, write the first `cap` entries only, leave everything behind
+    # them alone, and raise SAPS_ERR_OVERFLOW in the status word.
+    torch = torch_cuda()
+    n, p, lr, seed, cap = 6, 0.1, 0.05, 23, 4000
+    pairs_list = np.array([[1, 0, 2, 5, 4, 3], [5, 4, 3, 2, 1, 0], [0, 2, 1, 4, 3, 5]], dtype=np.int32)
+    x = synth.gaussian_matrix(n, N, 1.0, seed, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, seed, 1)
+    dx, dg = DeviceMatrix(x, ld), DeviceMatrix(g, ld)
+    ctx = sb.saps_create_ld(n, N, ld, seed)
+    sb.saps_set_pack_capacity(ctx, cap)
+    assert sb.saps_pack_capacity(ctx, p) == cap
+    guard = 64
+    vals = torch.full((n * cap + guard,), 123.0, dtype=torch.float32, device="cuda")
+    idx = torch.full((cap + guard,), -1, dtype=torch.int32, device="cuda")
+    T = len(pairs_list)
+    counts = torch.full((T + 1,), -1, dtype=torch.int32, device="cuda")
+    if scheduler:
+        sb.saps_run_rounds_pack(ctx, dx.ptr, dg.ptr, lr, 1, T, p, vals, idx, counts, pairs_list=pairs_list)
+    else:
+        for r in range(T):
+            sb.saps_round_pack(ctx, dx.ptr, dg.ptr, lr, pairs_list[r], 1 + r, p, vals, idx, counts[r:])
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == sb.SAPS_ERR_OVERFLOW
+    assert sb.saps_status(ctx) == 0                       # reading the status clears it
+    want = x.copy()
+    for r in range(T):
+        a = want.copy()
+        oracle.sgd(a, g, lr)
+        m = oracle.mask(seed, 1 + r, p, N)
+        wv, wi, wc = oracle.pack(a, m, cap)               # the oracle clamps the same way
+        oracle.pair_average(a, pairs_list[r], m)
+        want = a
+        assert wc > cap
+        assert int(counts[r]) == wc, f"round {r}: the true count is reported"
+    assert int(counts[T]) == -1
+    assert_bits_equal(dx.host(), want, "model after overflowing rounds")
+    gv, gi = vals.cpu().numpy(), idx.cpu().numpy().view(np.uint32)
+    assert (gi[:cap] == wi[:cap]).all() and (gi[cap:] == 0xFFFFFFFF).all()
+    assert_bits_equal(gv[:n * cap].reshape(n, cap), wv, "first cap entries of the last round's wire buffer")
+    assert (gv[n * cap:] == 123.0).all()
+    assert dx.canaries_intact() and dg.canaries_intact()
+    # with the formula capacity back, the same context emits a complete buffer again
+    sb.saps_set_pack_capacity(ctx, 0)
+    full = sb.saps_pack_capacity(ctx, p)
+    vals2 = torch.zeros(n, full, dtype=torch.float32, device="cuda")
+    idx2 = torch.zeros(full, dtype=torch.int32, device="cuda")
+    sb.saps_round_pack(ctx, dx.ptr, dg.ptr, lr, pairs_list[0], T + 1, p, vals2, idx2, counts)
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    a = want.copy()
+    oracle.sgd(a, g, lr)
+    m = oracle.mask(seed, T + 1, p, N)
+    wv, wi, wc = oracle.pack(a, m, full)
+    assert int(counts[0]) == wc <= full
+    assert (idx2.cpu().numpy().view(np.uint32)[:wc] == wi[:wc]).all()
+    assert_bits_equal(vals2.cpu().numpy()[:, :wc], wv[:, :wc], "wire buffer after the capacity was restored")
+    sb.saps_destroy(ctx)

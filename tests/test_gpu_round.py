@@ -239,11 +239,12 @@ def test_round_host_entry_point(sb):
     ld = round_up(N, 32)
     d_x = torch.empty(n * ld, dtype=torch.float32, device="cuda")
     d_g = torch.empty(n * ld, dtype=torch.float32, device="cuda")
-    ctx = sb.saps_create(n, N, 51)
+    ctx = sb.saps_create_ld(n, N, ld, 51)
     sb.saps_round_host(ctx, hx, hg, 0.05, pairs, 2, p, d_x, d_g)
     assert_bits_equal(hx.numpy(), want, "host entry point")
-    # without a gradient
+    # without a gradient, with many small chunks over all six lanes
     hx2 = torch.from_numpy(x.copy()).pin_memory()
+    sb.saps_set_host_pipeline(ctx, 100_000, 6)
     sb.saps_round_host(ctx, hx2, None, 0.0, pairs, 3, p, d_x, None)
     want2 = x.copy()
     oracle.gossip_round(want2, None, 0.0, pairs, 51, 3, p)
@@ -257,9 +258,9 @@ def test_round_pack_host_entry_point(sb):
     x = synth.gaussian_matrix(n, N, 0.05, 52, 0)
     g = synth.gaussian_matrix(n, N, 0.01, 52, 1)
     pairs = [1, 0, 3, 2, 5, 4]
-    ctx = sb.saps_create(n, N, 52)
-    cap = sb.saps_pack_capacity(ctx, p)
     ld = round_up(N, 32)
+    ctx = sb.saps_create_ld(n, N, ld, 52)
+    cap = sb.saps_pack_capacity(ctx, p)
     hx = torch.from_numpy(x.copy()).pin_memory()
     hg = torch.from_numpy(g).pin_memory()
     hv = torch.full((n, cap), 123.0, dtype=torch.float32).pin_memory()
@@ -283,8 +284,13 @@ def test_round_pack_host_entry_point(sb):
     assert (hi.numpy().view(np.uint32)[:wc] == wi[:wc]).all()
     assert_bits_equal(hv.numpy()[:, :wc], wv[:, :wc], "host wire buffer")
     assert_bits_equal(hx.numpy(), want, "host entry point with wire buffer")
-    # model resident on the device (x_host = NULL): only g goes in, the wire buffer comes out
-    ctx = sb.saps_create(n, N, 52)
+    # model resident on the device (x_host = NULL): only g goes in, the wire buffer comes out;
+    # one lane, and a row stride that only allows 64-bit accesses
+    ld = N + 2
+    d_x = torch.empty(n * ld, dtype=torch.float32, device="cuda")
+    d_g = torch.empty(n * ld, dtype=torch.float32, device="cuda")
+    ctx = sb.saps_create_ld(n, N, ld, 52)
+    sb.saps_set_host_pipeline(ctx, 4096, 1)
     d_x.view(n, ld)[:, :N].copy_(torch.from_numpy(x))
     sb.saps_round_pack_host(ctx, None, hg, 0.05, pairs, 4, p, d_x, d_g, hv, hi, hc, d_v, d_i, d_c)
     assert int(hc[0]) == wc
