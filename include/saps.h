@@ -37,7 +37,7 @@
  *   - The context owns small device scratch areas, each allocated by the first call that
  *     needs it, on the device that is current then (so such a first call must not happen
  *     inside a stream capture): the status word and the tile states of the compaction scan
- *     (16 + 12 ceil(N/2048) bytes; saps_pack and every emitting entry point), the per-tile
+ *     (16 + 8 ceil(N/2048) bytes; saps_pack and every emitting entry point), the per-tile
  *     counts and prefixes of the emitting round (12 ceil(N/2048) bytes), the partial sums of
  *     saps_consensus_distance (8 ceil(N/2048) bytes).  saps_round, saps_run_rounds,
  *     saps_mask, saps_unpack_avg* and saps_pack_noalloc allocate nothing.
@@ -205,7 +205,7 @@ SAPS_API int saps_unpack_avg_rows(saps_ctx* ctx, float* x, const float* recv_val
  * cudaMalloc nor cudaFree nor any library routine that does.
  *
  * Instead the tile states of the compaction scan live in a fixed array inside the library
- * image (786,448 bytes).  The CUDA runtime creates that array on a GPU when it loads the
+ * image (524,304 bytes).  The CUDA runtime creates that array on a GPU when it loads the
  * library's device code there (at the latest on the first launch of one of its kernels on
  * that GPU), not on demand from this call, and keeps it until the process exits.  That array covers N <= SAPS_NOALLOC_MAX_N columns; a larger context is refused
  * with SAPS_ERR_TOO_LARGE before anything is launched.

@@ -29,18 +29,16 @@ struct RowGroups {
 //   word 1            tile ticket of the running scan
 //   words 2..3        unused
 //   then ntiles x u64 tile states {flag << 32 | value}
-//   then ntiles x u32 exclusive prefix of every tile (kept for the fused emission)
 struct ScratchView {
     int* status;
     uint32_t* ticket;
     unsigned long long* tile_state;
-    uint32_t* tile_excl;
     uint32_t ntiles;
 };
 
 inline size_t scratch_bytes(uint32_t ntiles)
 {
-    return 16 + (size_t)ntiles * 8 + (size_t)ntiles * 4;
+    return 16 + (size_t)ntiles * 8;
 }
 
 inline ScratchView scratch_view(void* base, uint32_t ntiles)
@@ -50,7 +48,6 @@ inline ScratchView scratch_view(void* base, uint32_t ntiles)
     v.status = reinterpret_cast<int*>(p);
     v.ticket = reinterpret_cast<uint32_t*>(p + 4);
     v.tile_state = reinterpret_cast<unsigned long long*>(p + 16);
-    v.tile_excl = reinterpret_cast<uint32_t*>(p + 16 + (size_t)ntiles * 8);
     v.ntiles = ntiles;
     return v;
 }

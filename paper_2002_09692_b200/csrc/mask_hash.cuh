@@ -27,26 +27,33 @@ SAPS_HD uint32_t mix32(uint32_t v)
 }
 
 // Key of round t: what the coordinator would broadcast as the seed s (Algorithm 1).
+// k0f and k1f are the key words folded with their own upper halves, k ^ (k >> 16): the hash
+// xors a key word into v and then applies v ^= v >> 16, which equals xoring the folded word
+// into v ^ (v >> 16), one operation less per column.
 struct RoundKey {
-    uint32_t k0, k1;
+    uint32_t k0f, k1f;
     uint32_t thr32;   // low 32 bits of the threshold
     uint32_t all;     // 1 when the threshold is 2^32 (every column kept)
 };
 
-SAPS_HD uint32_t column_hash(uint32_t k, uint32_t k0, uint32_t k1)
+SAPS_HD uint32_t fold16(uint32_t w) { return w ^ (w >> 16); }
+
+// H(k): v = k ^ k0; v ^= v >> 16; v *= M1; v ^= v >> 15; v *= M2; v ^= k1; v ^= v >> 16;
+//       v *= M3; v ^= v >> 15, written with the folded key words.
+SAPS_HD uint32_t column_hash(uint32_t k, uint32_t k0f, uint32_t k1f)
 {
-    uint32_t v = k ^ k0;
-    v ^= v >> 16; v *= kMul1;
+    uint32_t v = k ^ (k >> 16) ^ k0f;
+    v *= kMul1;
     v ^= v >> 15; v *= kMul2;
-    v ^= k1;
-    v ^= v >> 16; v *= kMul3;
+    v = v ^ (v >> 16) ^ k1f;
+    v *= kMul3;
     v ^= v >> 15;
     return v;
 }
 
 SAPS_HD bool column_kept(uint32_t k, const RoundKey& key)
 {
-    return (column_hash(k, key.k0, key.k1) < key.thr32) | (key.all != 0);
+    return (column_hash(k, key.k0f, key.k1f) < key.thr32) | (key.all != 0);
 }
 
 }  // namespace saps

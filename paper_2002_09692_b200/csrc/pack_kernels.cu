@@ -14,9 +14,9 @@ namespace saps {
 namespace {
 
 // Scratch of the allocation-free compaction entry point: the same layout as a context's
-// scratch (status word, ticket, tile states, tile prefixes) for up to kStaticMaxTiles column
+// scratch (status word, ticket, tile states) for up to kStaticMaxTiles column
 // tiles.  Every GPU that loads the library holds these bytes until the process exits.
-__device__ __align__(256) unsigned char g_static_scratch[16 + (size_t)kStaticMaxTiles * 12];
+__device__ __align__(256) unsigned char g_static_scratch[16 + (size_t)kStaticMaxTiles * 8];
 
 constexpr unsigned long long kFlagAggregate = 1ull << 32;
 constexpr unsigned long long kFlagInclusive = 2ull << 32;
@@ -87,6 +87,16 @@ __device__ __forceinline__ bool lookback_exclusive(const ScratchView& sc, uint32
     return ok;
 }
 
+// One kept value of x.  A sparse gather touches one 32-byte sector per value; the qualifier
+// asks the L2 to fetch 64 bytes for it instead of the whole 128-byte line it would fetch by
+// default, which halves the DRAM traffic of the gather (there is no smaller request size).
+__device__ __forceinline__ float load_gather(const float* p)
+{
+    float v;
+    asm volatile("ld.global.nc.L2::64B.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+
 template <bool GATHER>
 __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
 {
@@ -94,7 +104,7 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
     constexpr int kSteps = kTileCols / kThreads;  // ballots per warp
     __shared__ uint32_t s_tile, s_excl, s_abort;
     __shared__ uint32_t s_warp_cnt[kWarps];
-    __shared__ uint32_t s_kept[kTileCols];
+    __shared__ uint16_t s_kept[kTileCols];        // kept columns as offsets inside the tile
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
@@ -106,15 +116,27 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
     if (tile >= a.scratch.ntiles) return;  // cannot happen with a cleared ticket; stay in bounds
 
     // ---- mask words of this warp's 8 x 32 columns ----
-    const uint64_t col_warp = (uint64_t)tile * kTileCols + (uint64_t)warp * (32 * kSteps);
+    // 32-bit column arithmetic: N < 2^32, so the tile's first column fits, and `rem` is the
+    // number of columns from there to the end of the row.  The hash input of a column beyond
+    // the row may wrap; it is masked by the bounds test.
+    const uint32_t col0 = tile * (uint32_t)kTileCols;
+    const uint32_t rem = a.N - col0;
+    const uint32_t off0 = (uint32_t)warp * (32 * kSteps) + lane;
+    const uint32_t hash0 = a.col_offset + col0 + off0;
     uint32_t word[kSteps];
     uint32_t cnt = 0;
+    if (rem >= (uint32_t)kTileCols) {
 #pragma unroll
-    for (int s = 0; s < kSteps; ++s) {
-        const uint64_t k = col_warp + s * 32 + lane;
-        const bool kept = (k < a.N) && column_kept(a.col_offset + (uint32_t)k, a.key);
-        word[s] = __ballot_sync(0xFFFFFFFFu, kept);
-        cnt += __popc(word[s]);
+        for (int s = 0; s < kSteps; ++s) {
+            word[s] = __ballot_sync(0xFFFFFFFFu, column_kept(hash0 + s * 32, a.key));
+            cnt += __popc(word[s]);
+        }
+    } else {
+#pragma unroll
+        for (int s = 0; s < kSteps; ++s) {
+            word[s] = __ballot_sync(0xFFFFFFFFu, (off0 + s * 32 < rem) && column_kept(hash0 + s * 32, a.key));
+            cnt += __popc(word[s]);
+        }
     }
     if (lane == 0) s_warp_cnt[warp] = cnt;
     __syncthreads();
@@ -131,49 +153,46 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
         uint32_t excl;
         const bool ok = lookback_exclusive(a.scratch, tile, total, a.spin_limit, a.skip_tile, lane, &excl);
         if (lane == 0) {
-            if (ok) {
-                a.scratch.tile_excl[tile] = excl;
+            if (ok)
                 s_excl = excl;
-            } else {
+            else
                 s_abort = 1;
-            }
         }
+    }
+
+    // ---- the tile's kept columns, ascending, to shared memory (this needs no prefix) ----
+    const uint32_t below = (1u << lane) - 1u;
+    uint32_t r = warp_off;
+#pragma unroll
+    for (int s = 0; s < kSteps; ++s) {
+        if ((word[s] >> lane) & 1u) s_kept[r + __popc(word[s] & below)] = (uint16_t)(off0 + s * 32);
+        r += __popc(word[s]);
     }
     __syncthreads();
     if (s_abort) return;
     const uint32_t base = s_excl;
 
-    // ---- the tile's kept columns, ascending, to shared memory and to out_idx ----
-    uint32_t r = warp_off;
-#pragma unroll
-    for (int s = 0; s < kSteps; ++s) {
-        if ((word[s] >> lane) & 1u) {
-            const uint32_t mine = r + __popc(word[s] & ((1u << lane) - 1u));
-            const uint32_t k = (uint32_t)(col_warp + s * 32 + lane);
-            s_kept[mine] = k;
-            if (a.out_idx != nullptr && base + mine < a.cap) a.out_idx[base + mine] = a.col_offset + k;
-        }
-        r += __popc(word[s]);
-    }
-
     if (tile == a.scratch.ntiles - 1 && tid == 0) {
         if (a.out_count != nullptr) *a.out_count = base + total;
         if (base + total > a.cap) atomicCAS(a.scratch.status, 0, -4 /* SAPS_ERR_OVERFLOW */);
     }
+    if (total == 0) return;
+    const uint32_t room = base < a.cap ? a.cap - base : 0u;
+    const uint32_t take = total < room ? total : room;
+    if (a.out_idx != nullptr)
+        for (uint32_t q = tid; q < take; q += kThreads) a.out_idx[base + q] = a.col_offset + col0 + s_kept[q];
 
     // ---- gather: only the kept lanes of x are ever loaded ----
     if constexpr (GATHER) {
-        __syncthreads();
-        if (total == 0) return;
-        const uint32_t room = base < a.cap ? a.cap - base : 0u;
-        const uint32_t take = total < room ? total : room;
         // one flat loop over (worker, kept column): with a sparse mask a tile keeps only a few
         // columns, so looping over workers inside keeps every thread busy and all the
         // (uncoalesced, sector-sized) loads of a tile in flight at once
+        const float* xt = a.x + col0;
         const uint32_t items = (uint32_t)a.n * take;
+#pragma unroll 4
         for (uint32_t e = tid; e < items; e += kThreads) {
             const uint32_t i = e / take, q = e - i * take;
-            a.out_vals[(size_t)i * a.cap + base + q] = __ldg(a.x + (size_t)i * a.ld + s_kept[q]);
+            a.out_vals[(size_t)i * a.cap + base + q] = load_gather(xt + (size_t)i * a.ld + s_kept[q]);
         }
     }
 }
@@ -269,6 +288,21 @@ __global__ void __launch_bounds__(kThreads) unpack_avg_kernel(const UnpackArgs a
 // Consensus distance, one block per column tile.  Per column the deviations are taken from
 // worker 0's value (exact in fp64), sum d^2 - (sum d)^2 / n, so that identical workers give
 // exactly zero and nearly identical ones lose no digits.  VEC = 4 streams 128-bit vectors.
+// The kernel is a pure read stream: every thread first issues the loads of a batch of kRowBatch
+// workers (independent 16-byte loads, all in flight together), then accumulates them.
+constexpr int kRowBatch = 8;
+
+template <int VEC>
+__device__ __forceinline__ void load_row_chunk(const float* p, float (&v)[VEC])
+{
+    if constexpr (VEC == 4) {
+        const float4 q = __ldcs(reinterpret_cast<const float4*>(p));
+        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+    } else {
+        v[0] = __ldcs(p);
+    }
+}
+
 template <int VEC>
 __global__ void __launch_bounds__(kThreads) consensus_partial_kernel(const float* __restrict__ x, size_t ld,
                                                                      uint32_t N, int n, double* partials)
@@ -279,37 +313,47 @@ __global__ void __launch_bounds__(kThreads) consensus_partial_kernel(const float
     double acc = 0.0;
     const uint64_t col0 = (uint64_t)blockIdx.x * kTileCols;
     const uint32_t nfull = (VEC == 4) ? (N & ~3u) : N;
-#pragma unroll
+    const double inv_n = 1.0 / (double)n;
+#pragma unroll 1
     for (int u = 0; u < U; ++u) {
         const uint64_t k = col0 + (uint64_t)(u * kThreads + tid) * VEC;
         if (k < nfull) {
+            const float* col = x + k;
+            float first[VEC];
+            load_row_chunk<VEC>(col, first);
             double pivot[VEC], sd[VEC], sdd[VEC];
-            if constexpr (VEC == 4) {
-                const float4 p = __ldcs(reinterpret_cast<const float4*>(x + k));
-                pivot[0] = p.x; pivot[1] = p.y; pivot[2] = p.z; pivot[3] = p.w;
-            } else {
-                pivot[0] = __ldcs(x + k);
-            }
 #pragma unroll
-            for (int c = 0; c < VEC; ++c) sd[c] = sdd[c] = 0.0;
-#pragma unroll 4
-            for (int i = 1; i < n; ++i) {
-                float v[VEC];
-                if constexpr (VEC == 4) {
-                    const float4 q = __ldcs(reinterpret_cast<const float4*>(x + (size_t)i * ld + k));
-                    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
-                } else {
-                    v[0] = __ldcs(x + (size_t)i * ld + k);
+            for (int c = 0; c < VEC; ++c) {
+                pivot[c] = (double)first[c];
+                sd[c] = sdd[c] = 0.0;
+            }
+            int i = 1;
+            for (; i + kRowBatch <= n; i += kRowBatch) {
+                float v[kRowBatch][VEC];
+#pragma unroll
+                for (int b = 0; b < kRowBatch; ++b) load_row_chunk<VEC>(col + (size_t)(i + b) * ld, v[b]);
+#pragma unroll
+                for (int b = 0; b < kRowBatch; ++b) {
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c) {
+                        const double d = (double)v[b][c] - pivot[c];
+                        sd[c] += d;
+                        sdd[c] = __fma_rn(d, d, sdd[c]);
+                    }
                 }
+            }
+            for (; i < n; ++i) {
+                float v[VEC];
+                load_row_chunk<VEC>(col + (size_t)i * ld, v);
 #pragma unroll
                 for (int c = 0; c < VEC; ++c) {
                     const double d = (double)v[c] - pivot[c];
                     sd[c] += d;
-                    sdd[c] += d * d;
+                    sdd[c] = __fma_rn(d, d, sdd[c]);
                 }
             }
 #pragma unroll
-            for (int c = 0; c < VEC; ++c) acc += sdd[c] - sd[c] * sd[c] / (double)n;
+            for (int c = 0; c < VEC; ++c) acc += sdd[c] - sd[c] * sd[c] * inv_n;
         }
     }
     if constexpr (VEC == 4) {
@@ -321,9 +365,9 @@ __global__ void __launch_bounds__(kThreads) consensus_partial_kernel(const float
             for (int i = 1; i < n; ++i) {
                 const double d = (double)x[(size_t)i * ld + k] - pivot;
                 sd += d;
-                sdd += d * d;
+                sdd = __fma_rn(d, d, sdd);
             }
-            acc += sdd - sd * sd / (double)n;
+            acc += sdd - sd * sd * inv_n;
         }
     }
 #pragma unroll

@@ -62,7 +62,10 @@ uint64_t threshold64(double keep_frac)
 RoundKey make_key(uint64_t seed, uint64_t t, double keep_frac)
 {
     RoundKey key;
-    saps_round_key(seed, t, &key.k0, &key.k1);
+    uint32_t k0 = 0, k1 = 0;
+    saps_round_key(seed, t, &k0, &k1);
+    key.k0f = fold16(k0);
+    key.k1f = fold16(k1);
     const uint64_t thr = threshold64(keep_frac);
     key.all = thr >= (1ull << 32) ? 1u : 0u;
     key.thr32 = key.all ? 0xFFFFFFFFu : (uint32_t)thr;
