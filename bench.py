@@ -3,8 +3,8 @@
 
 One step = one pass of the whole hot path for one round t: peer selection on the host
 (Algorithm 3), then on the GPU the SGD step, the round mask, the emission of the packed
-wire buffer and the pair average (saps_round_pack: a mask-scan kernel and the fused round
-kernel).  Inputs are synthetic Gaussian fp32 matrices of the configured size, resident in
+wire buffer and the pair average (saps_round_pack: one fused kernel per round, which also
+counts the next round's mask).  Inputs are synthetic Gaussian fp32 matrices of the configured size, resident in
 HBM when the timed region starts.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload vgg16] [--keep-frac 0.01]
@@ -336,12 +336,12 @@ def run_ours(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": dict(workload_config(w, p, world),
-                       gpu_step="saps_select_peers + saps_round_pack (tile prefix-scan kernel + fused "
-                                "SGD/mask/emit/average kernel, which also counts the next round's mask per tile)"),
+                       gpu_step="saps_select_peers + saps_round_pack (one fused SGD/mask/emit/average kernel per step; "
+                                "it also counts the next round's mask per tile, so no separate scan runs)"),
         "effective_hbm_gbs": bytes_round * K / (elapsed_ms * 1e-3) / 1e9,
         "frac_of_8tbs": bytes_round * K / (elapsed_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
         "kept_columns": kept,
-        "gpu_launches": 2 * K,
+        "gpu_launches": K,
         "clocks": clocks,
         "roofline": {
             "bound": "hbm" if 2 * 4 * n * N >= L2_BYTES else "l2-resident",

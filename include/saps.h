@@ -38,8 +38,8 @@
  *     needs it, on the device that is current then (so such a first call must not happen
  *     inside a stream capture): the status word and the tile states of the compaction scan
  *     (16 + 8 ceil(N/2048) bytes; saps_pack and every emitting entry point), the per-tile
- *     counts and prefixes of the emitting round (12 ceil(N/2048) bytes), the partial sums of
- *     saps_consensus_distance (8 ceil(N/2048) bytes).  saps_round, saps_run_rounds,
+ *     and per-group mask counts of the emitting round (about 8 ceil(N/2048) bytes), the partial sums of
+ *     saps_consensus_distance (8 ceil(N/1024) bytes).  saps_round, saps_run_rounds,
  *     saps_mask, saps_unpack_avg* and saps_pack_noalloc allocate nothing.
  *   - Calls on one context must not overlap on the GPU (use one stream, or order streams
  *     with events): they share the scratch area.
@@ -127,10 +127,11 @@ SAPS_API int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, 
                     uint32_t* out_count, void* stream);
 
 /* The emitting entry points need the number of kept columns per column tile before the fused
- * kernel runs.  By default that kernel also counts them for round t+1 while it streams round
- * t (the mask does not depend on the data, and the integer units are idle in a memory-bound
- * kernel), so a following call for round t+1 with the same keep_frac only has to take a
- * prefix sum of a few thousand numbers.  Any other call counts in a kernel of its own.
+ * kernel runs (a block derives the ranks of its kept columns from the counts of all earlier
+ * tiles).  By default that kernel also counts them for round t+1 while it streams round t (the
+ * mask does not depend on the data, and the integer units are not the bottleneck of a
+ * memory-bound kernel), so a following call for round t+1 with the same keep_frac is a single
+ * kernel launch.  Any other call first counts in a small kernel of its own.
  * Results are identical either way; enabled = 0 switches the run-ahead off.
  * The counts are kept in the context and read by the next call's kernels, so consecutive
  * emitting calls on one context must run on one stream or be ordered by events (the general
@@ -320,7 +321,9 @@ SAPS_API int saps_set_host_pipeline(saps_ctx* ctx, uint64_t chunk_columns, int l
 /* Consensus distance of Theorem 1 / Lemma 2: *out = || X - Xbar 1^T ||_F^2, the sum over all
  * coordinates of the squared deviations of the n workers from their mean, accumulated in
  * fp64 in a fixed order (the result is reproducible).  x: device [n, ld]; out: device, one
- * double.  Reads x once.  The first call allocates ceil(N/2048) doubles of scratch. */
+ * double.  Reads x once: every block of 1024 columns leaves a partial sum, and a one-block kernel,
+ * launched so that it is already in place when the first one ends, adds them up.  The first call
+ * allocates ceil(N/1024) doubles. */
 SAPS_API int saps_consensus_distance(saps_ctx* ctx, const float* x, double* out, void* stream);
 
 /* Host only.  Communication figures of one round (Table 1; the bandwidth utilisation of

@@ -72,14 +72,25 @@ struct RoundArgs {
     uint32_t tile_begin;   // first column tile to process
     uint32_t tile_count;   // number of column tiles to process
     int gossip_first;      // 0: Algorithm 2's order (SGD, then average); 1: Eq. 7's order
-    // emission of the wire buffer (all NULL/0 when not emitting)
+    // emission of the wire buffer (all NULL/0 when not emitting).  The ranks of a tile's kept
+    // columns start at the number of kept columns in all earlier tiles.  That number is summed by
+    // the block itself from two small arrays: the kept columns per tile, and their sums over
+    // groups of 2^group_shift consecutive tiles.
     float* out_vals;
     uint32_t cap;
-    const uint32_t* tile_excl;   // exclusive prefix of kept columns per tile
+    const uint32_t* tile_cnt;    // kept columns per tile, this round
+    const uint32_t* group_cnt;   // the same summed over every group of tiles
+    uint32_t group_shift;
+    uint32_t ngroups;
     uint32_t* out_idx;           // kept columns, written by the first row group (may be NULL)
-    // run-ahead for the next round: the first row group also counts, per tile, the columns
-    // that the NEXT round's mask keeps (NULL = off)
+    uint32_t* out_count;         // total, written by the block of tile 0 (may be NULL)
+    int* status;                 // receives SAPS_ERR_OVERFLOW when the total exceeds cap
+    // run-ahead for the next round: the first row group also counts, per tile and per group, the
+    // columns that the NEXT round's mask keeps (NULL = off), and clears the group sums that the
+    // round after next will accumulate into
     uint32_t* next_cnt;
+    uint32_t* next_group_cnt;
+    uint32_t* clear_group_cnt;
     RoundKey next_key;
 };
 
@@ -103,12 +114,10 @@ struct PackArgs {
 
 cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream);
 
-// Mask scan without model data, in two small steps: kept columns per tile, then their
-// exclusive prefix, the total (out_count, may be NULL) and the overflow check.
+// Mask scan without model data: kept columns per tile, added up per group of 2^group_shift tiles
+// as well (group_cnt must be zero before).
 cudaError_t launch_mask_count(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t ntiles, uint32_t* tile_cnt,
-                              cudaStream_t stream);
-cudaError_t launch_tile_scan(const uint32_t* tile_cnt, uint32_t ntiles, uint32_t* tile_excl, uint32_t* out_count,
-                             uint32_t cap, int* status, cudaStream_t stream);
+                              uint32_t* group_cnt, uint32_t group_shift, cudaStream_t stream);
 
 cudaError_t launch_mask(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t* out_bits,
                         cudaStream_t stream);
@@ -128,9 +137,12 @@ struct UnpackArgs {
 };
 cudaError_t launch_unpack_avg(const UnpackArgs& a, cudaStream_t stream);
 
-// || X - mean over workers ||_F^2: per-tile partial sums, then one block adds them in order.
-cudaError_t launch_consensus(const float* x, size_t ld, uint32_t N, int n, uint32_t ntiles,
-                             double* partials, double* out, cudaStream_t stream);
+// || X - mean over workers ||_F^2: one partial sum per block of kConsensusCols columns
+// (consensus_blocks(N) doubles), then a one-block kernel adds them in a fixed order.
+constexpr int kConsensusCols = 1024;
+inline uint32_t consensus_blocks(uint32_t N) { return (uint32_t)(((uint64_t)N + kConsensusCols - 1) / kConsensusCols); }
+cudaError_t launch_consensus(const float* x, size_t ld, uint32_t N, int n, double* partials, double* out,
+                             cudaStream_t stream);
 
 // Compaction on the library's static scratch area (no allocation anywhere on the path).
 constexpr uint32_t kStaticMaxTiles = 65536;  // kTileCols columns each: N <= 134,217,728

@@ -199,7 +199,8 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
 
 // Kept columns of every tile under one round's mask (no model data): one warp per tile.
 __global__ void __launch_bounds__(kThreads) mask_count_kernel(uint32_t N, uint32_t col_offset, RoundKey key,
-                                                             uint32_t ntiles, uint32_t* tile_cnt)
+                                                             uint32_t ntiles, uint32_t* tile_cnt, uint32_t* group_cnt,
+                                                             uint32_t group_shift)
 {
     const int lane = threadIdx.x & 31;
     const uint32_t tile = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
@@ -212,52 +213,9 @@ __global__ void __launch_bounds__(kThreads) mask_count_kernel(uint32_t N, uint32
         cnt += ((k < N) && column_kept(col_offset + (uint32_t)k, key)) ? 1u : 0u;
     }
     cnt = warp_sum(cnt);
-    if (lane == 0) tile_cnt[tile] = cnt;
-}
-
-// Exclusive prefix of the tile counts, the total and the overflow check, by one block: every
-// thread owns a contiguous run of tiles (a handful for tens of millions of columns), sums it,
-// the block scans the 1024 sums once, and every thread writes the prefixes of its run.
-constexpr int kScanThreads = 1024;
-__global__ void __launch_bounds__(kScanThreads) tile_scan_kernel(const uint32_t* __restrict__ tile_cnt,
-                                                                 uint32_t ntiles, uint32_t* __restrict__ tile_excl,
-                                                                 uint32_t* out_count, uint32_t cap, int* status)
-{
-    __shared__ uint32_t s_warp[kScanThreads / 32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t per = (ntiles + kScanThreads - 1) / kScanThreads;
-    const uint64_t lo64 = (uint64_t)tid * per;
-    const uint32_t lo = lo64 < ntiles ? (uint32_t)lo64 : ntiles;
-    const uint32_t hi = lo64 + per < ntiles ? (uint32_t)(lo64 + per) : ntiles;
-    uint32_t mine = 0;
-    for (uint32_t i = lo; i < hi; ++i) mine += tile_cnt[i];
-    uint32_t inc = mine;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-        if (lane >= d) inc += o;
-    }
-    if (lane == 31) s_warp[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        uint32_t w = s_warp[lane];
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, w, d);
-            if (lane >= d) w += o;
-        }
-        s_warp[lane] = w;  // inclusive over warps
-    }
-    __syncthreads();
-    uint32_t run = (warp ? s_warp[warp - 1] : 0u) + inc - mine;
-    for (uint32_t i = lo; i < hi; ++i) {
-        tile_excl[i] = run;
-        run += tile_cnt[i];
-    }
-    if (tid == kScanThreads - 1) {
-        const uint32_t total = s_warp[kScanThreads / 32 - 1];
-        if (out_count != nullptr) *out_count = total;
-        if (total > cap) atomicCAS(status, 0, -4 /* SAPS_ERR_OVERFLOW */);
+    if (lane == 0) {
+        tile_cnt[tile] = cnt;
+        atomicAdd(group_cnt + (tile >> group_shift), cnt);
     }
 }
 
@@ -285,7 +243,8 @@ __global__ void __launch_bounds__(kThreads) unpack_avg_kernel(const UnpackArgs a
     *p = __fmul_rn(0.5f, __fadd_rn(*p, __ldg(a.recv + (size_t)src * a.cap + r)));
 }
 
-// Consensus distance, one block per column tile.  Per column the deviations are taken from
+// Consensus distance, one block per kConsensusCols columns (half a column tile: blocks this
+// small keep the last, partly filled wave of the grid short).  Per column the deviations are taken from
 // worker 0's value (exact in fp64), sum d^2 - (sum d)^2 / n, so that identical workers give
 // exactly zero and nearly identical ones lose no digits.  VEC = 4 streams 128-bit vectors.
 // The kernel is a pure read stream: every thread first issues the loads of a batch of kRowBatch
@@ -304,14 +263,17 @@ __device__ __forceinline__ void load_row_chunk(const float* p, float (&v)[VEC])
 }
 
 template <int VEC>
-__global__ void __launch_bounds__(kThreads) consensus_partial_kernel(const float* __restrict__ x, size_t ld,
-                                                                     uint32_t N, int n, double* partials)
+__global__ void __launch_bounds__(kThreads) consensus_kernel(const float* __restrict__ x, size_t ld, uint32_t N, int n,
+                                                             double* partials)
 {
-    constexpr int U = kTileCols / (kThreads * VEC);
+    constexpr int U = kConsensusCols / (kThreads * VEC);
     __shared__ double s_part[kThreads / 32];
     const int tid = threadIdx.x;
+    // the kernel that adds up the partial sums may be set up while this one still runs; it waits
+    // for this grid to complete before it reads anything
+    cudaTriggerProgrammaticLaunchCompletion();
     double acc = 0.0;
-    const uint64_t col0 = (uint64_t)blockIdx.x * kTileCols;
+    const uint64_t col0 = (uint64_t)blockIdx.x * kConsensusCols;
     const uint32_t nfull = (VEC == 4) ? (N & ~3u) : N;
     const double inv_n = 1.0 / (double)n;
 #pragma unroll 1
@@ -358,7 +320,7 @@ __global__ void __launch_bounds__(kThreads) consensus_partial_kernel(const float
     }
     if constexpr (VEC == 4) {
         // the last (N mod 4) columns
-        if ((uint32_t)tid < N - nfull && col0 <= nfull && nfull < col0 + kTileCols) {
+        if ((uint32_t)tid < N - nfull && col0 <= nfull && nfull < col0 + kConsensusCols) {
             const uint32_t k = nfull + tid;  // cannot wrap: tid < N - nfull
             const double pivot = (double)x[k];
             double sd = 0.0, sdd = 0.0;
@@ -381,19 +343,33 @@ __global__ void __launch_bounds__(kThreads) consensus_partial_kernel(const float
     }
 }
 
-__global__ void __launch_bounds__(kThreads) consensus_final_kernel(const double* partials, uint32_t count,
-                                                                   double* out)
+// Adds the partial sums in a fixed order (the result is reproducible).  Launched so that it may
+// start before the kernel above has finished: everything it reads comes after the wait.
+constexpr int kFinalThreads = 1024;
+__global__ void __launch_bounds__(kFinalThreads) consensus_final_kernel(const double* partials, uint32_t count,
+                                                                        double* out)
 {
-    __shared__ double s_part[kThreads];
-    double acc = 0.0;
-    for (uint32_t i = threadIdx.x; i < count; i += kThreads) acc += partials[i];
-    s_part[threadIdx.x] = acc;
+    __shared__ double s_sum[kFinalThreads];
+    const uint32_t tid = threadIdx.x;
+    cudaGridDependencySynchronize();
+    // eight loads in flight per thread; the order of the additions is fixed all the same
+    double sum = 0.0;
+    uint32_t i = tid;
+    for (; i + 7 * kFinalThreads < count; i += 8 * kFinalThreads) {
+        double v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = __ldcg(partials + i + j * kFinalThreads);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sum += v[j];
+    }
+    for (; i < count; i += kFinalThreads) sum += __ldcg(partials + i);
+    s_sum[tid] = sum;
     __syncthreads();
-    for (int d = kThreads / 2; d > 0; d >>= 1) {
-        if ((int)threadIdx.x < d) s_part[threadIdx.x] += s_part[threadIdx.x + d];
+    for (uint32_t d = kFinalThreads / 2; d > 0; d >>= 1) {
+        if (tid < d) s_sum[tid] += s_sum[tid + d];
         __syncthreads();
     }
-    if (threadIdx.x == 0) *out = s_part[0] < 0.0 ? 0.0 : s_part[0];
+    if (tid == 0) *out = s_sum[0] < 0.0 ? 0.0 : s_sum[0];
 }
 
 }  // namespace
@@ -406,17 +382,29 @@ cudaError_t launch_unpack_avg(const UnpackArgs& a, cudaStream_t stream)
     return cudaGetLastError();
 }
 
-cudaError_t launch_consensus(const float* x, size_t ld, uint32_t N, int n, uint32_t ntiles, double* partials,
-                             double* out, cudaStream_t stream)
+cudaError_t launch_consensus(const float* x, size_t ld, uint32_t N, int n, double* partials, double* out,
+                             cudaStream_t stream)
 {
+    const uint32_t blocks = consensus_blocks(N);
     if (ld % 4 == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0)
-        consensus_partial_kernel<4><<<ntiles, kThreads, 0, stream>>>(x, ld, N, n, partials);
+        consensus_kernel<4><<<blocks, kThreads, 0, stream>>>(x, ld, N, n, partials);
     else
-        consensus_partial_kernel<1><<<ntiles, kThreads, 0, stream>>>(x, ld, N, n, partials);
+        consensus_kernel<1><<<blocks, kThreads, 0, stream>>>(x, ld, N, n, partials);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    consensus_final_kernel<<<1, kThreads, 0, stream>>>(partials, ntiles, out);
-    return cudaGetLastError();
+    // programmatic dependent launch: the one-block summation is scheduled while the first kernel
+    // drains, which removes the launch gap between the two
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1, 1, 1);
+    cfg.blockDim = dim3(kFinalThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, consensus_final_kernel, (const double*)partials, blocks, out);
 }
 
 cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream)
@@ -470,18 +458,11 @@ cudaError_t launch_pack_static(PackArgs a, uint32_t ntiles, int* out_status, cud
 }
 
 cudaError_t launch_mask_count(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t ntiles, uint32_t* tile_cnt,
-                              cudaStream_t stream)
+                              uint32_t* group_cnt, uint32_t group_shift, cudaStream_t stream)
 {
     const uint32_t per_block = kThreads / 32;
     mask_count_kernel<<<(ntiles + per_block - 1) / per_block, kThreads, 0, stream>>>(N, col_offset, key, ntiles,
-                                                                                    tile_cnt);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_tile_scan(const uint32_t* tile_cnt, uint32_t ntiles, uint32_t* tile_excl, uint32_t* out_count,
-                             uint32_t cap, int* status, cudaStream_t stream)
-{
-    tile_scan_kernel<<<1, kScanThreads, 0, stream>>>(tile_cnt, ntiles, tile_excl, out_count, cap, status);
+                                                                                    tile_cnt, group_cnt, group_shift);
     return cudaGetLastError();
 }
 

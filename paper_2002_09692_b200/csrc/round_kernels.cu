@@ -89,10 +89,6 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
     const uint32_t nfull = a.N - a.N % VEC;
     const uint64_t col_tile = (uint64_t)tile * kTileCols;
 
-    // the tile's rank offset is asked for first, so that its latency hides under the model loads
-    uint32_t excl = 0;
-    if constexpr (EMIT) excl = __ldg(a.tile_excl + tile);
-
     Chunk<VEC> va[U], vb[U], wa[U], wb[U];
     bool inb[U];
     uint32_t col[U];
@@ -110,6 +106,17 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
                 if (HAS_G) wb[u] = load_stream<VEC>(gb + k);
             }
         }
+    }
+
+    // The rank offset of the tile = kept columns in all earlier tiles: whole groups of tiles from
+    // the group sums, the rest tile by tile; every thread takes a share (one load, seldom more),
+    // the block adds them up further down.  Placed behind the model loads, so that waiting for
+    // these few values never delays them.
+    uint32_t excl_part = 0;
+    if constexpr (EMIT) {
+        const uint32_t g = tile >> a.group_shift;
+        for (uint32_t j = tid; j < g; j += kThreads) excl_part += __ldg(a.group_cnt + j);
+        for (uint32_t j = (g << a.group_shift) + tid; j < tile; j += kThreads) excl_part += __ldg(a.tile_cnt + j);
     }
 
     uint32_t bits[U];
@@ -132,9 +139,15 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
 
     uint32_t rank[U];       // EMIT only: rank of this thread's first kept column
     uint32_t total = 0;     // EMIT only: kept columns in the vector part of the tile
+    uint32_t excl = 0;      // EMIT only: kept columns in all earlier tiles
     if constexpr (EMIT) {
         __shared__ uint32_t s_warp[U][kWarps];
+        __shared__ uint32_t s_excl[32];
         const int lane = tid & 31, warp = tid >> 5;
+        {
+            const uint32_t e = __reduce_add_sync(0xFFFFFFFFu, excl_part);
+            if (lane == 0) s_excl[warp] = e;
+        }
         uint32_t within[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -144,6 +157,7 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
             if (lane == 31) s_warp[u][warp] = inc;
         }
         __syncthreads();
+        excl = __reduce_add_sync(0xFFFFFFFFu, lane < kWarps ? s_excl[lane] : 0u);
         uint32_t running = excl;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -198,6 +212,7 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
 #pragma unroll
                 for (int w = 0; w < kWarps; ++w) t += s_next[w];
                 a.next_cnt[tile] = t;
+                atomicAdd(a.next_group_cnt + (tile >> a.group_shift), t);
             }
         }
         // what each worker sends: its value before the average (post-SGD in Algorithm 2's order)
@@ -290,6 +305,29 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
             } else if (HAS_G) {
                 xa[k] = pa;
             }
+        }
+    }
+
+    // once per round, by the block of tile 0: the total of kept columns, the overflow report,
+    // and clean group sums for the round after next
+    if constexpr (EMIT) {
+        if (tile == 0 && blockIdx.y == 0) {
+            __shared__ uint32_t s_tot[kWarps];
+            uint32_t t = 0;
+            for (uint32_t j = tid; j < a.ngroups; j += kThreads) t += __ldg(a.group_cnt + j);
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, d);
+            if ((tid & 31) == 0) s_tot[tid >> 5] = t;
+            __syncthreads();
+            if (tid == 0) {
+                uint32_t sum = 0;
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) sum += s_tot[w];
+                if (a.out_count != nullptr) *a.out_count = sum;
+                if (sum > a.cap) atomicCAS(a.status, 0, -4 /* SAPS_ERR_OVERFLOW */);
+            }
+            if (a.clear_group_cnt != nullptr)
+                for (uint32_t j = tid; j < a.ngroups; j += kThreads) a.clear_group_cnt[j] = 0;
         }
     }
 }

@@ -21,7 +21,7 @@ struct saps_ctx {
     int gossip_first;       // update order: 0 Algorithm 2, 1 Eq. 7
     uint32_t spin_limit;    // poll budget of the look-back
     uint32_t skip_tile;     // test hook, 0xFFFFFFFF = off
-    double* partials;       // device, ntiles doubles, for the consensus distance
+    double* partials;       // device, for the consensus distance: one double per block of columns
     uint64_t cap_override;  // 0 = capacity from the binomial bound
     // device scratch, allocated on first use on the then-current device
     void* scratch;
@@ -36,10 +36,14 @@ struct saps_ctx {
     bool lanes_ready;
     int host_lanes;             // lanes in use
     uint32_t host_chunk_tiles;  // column tiles per chunk
-    // Mask scan of the emitting round (saps_round_pack): kept columns per tile for the current
-    // round and, counted ahead by the fused kernel itself, for the next one; their prefix.
-    uint32_t* emit_mem;        // device: cnt[0][ntiles], cnt[1][ntiles], excl[ntiles]
+    // Mask counts of the emitting round (saps_round_pack): kept columns per tile, and per group
+    // of 2^group_shift tiles, for the current round and, counted ahead by the fused kernel
+    // itself, for the next one.  The group sums rotate over three buffers: read this round,
+    // accumulated for the next round, cleared for the round after.
+    uint32_t* emit_mem;        // device: cnt[2][ntiles], group_cnt[3][ngroups]
+    uint32_t group_shift, ngroups;
     int emit_cur;              // which cnt buffer the next call looks at
+    int group_cur;             // which group_cnt buffer the next call looks at
     bool ahead_valid;          // cnt[emit_cur] holds the counts of round ahead_t ...
     uint64_t ahead_t, ahead_thr;
     uint32_t ahead_col_offset; // ... for this threshold and column offset
@@ -155,9 +159,16 @@ RoundArgs round_args(const saps_ctx* ctx, float* x, const float* g, float lr, co
     a.gossip_first = ctx->gossip_first;
     a.out_vals = nullptr;
     a.cap = 0;
-    a.tile_excl = nullptr;
+    a.tile_cnt = nullptr;
+    a.group_cnt = nullptr;
+    a.group_shift = ctx->group_shift;
+    a.ngroups = ctx->ngroups;
     a.out_idx = nullptr;
+    a.out_count = nullptr;
+    a.status = nullptr;
     a.next_cnt = nullptr;
+    a.next_group_cnt = nullptr;
+    a.clear_group_cnt = nullptr;
     a.next_key = key;
     return a;
 }
@@ -212,6 +223,11 @@ int saps_create_ld(int n, uint64_t N, uint64_t ld, uint64_t seed, saps_ctx** out
     ctx->host_chunk_tiles = 512;
     ctx->emit_mem = nullptr;
     ctx->emit_cur = 0;
+    ctx->group_cur = 0;
+    // groups of about sqrt(ntiles) tiles: a block then adds up at most about 2 sqrt(ntiles) numbers
+    ctx->group_shift = 0;
+    while ((1ull << (2 * ctx->group_shift)) < ctx->ntiles) ++ctx->group_shift;
+    ctx->ngroups = (ctx->ntiles + (1u << ctx->group_shift) - 1) >> ctx->group_shift;
     ctx->ahead_valid = false;
     ctx->ahead_t = ctx->ahead_thr = 0;
     ctx->ahead_col_offset = 0;
@@ -360,13 +376,13 @@ int saps_consensus_distance(saps_ctx* ctx, const float* x, double* out, void* st
     if (ctx == nullptr || x == nullptr || out == nullptr) return SAPS_ERR_INVALID;
     if (ctx->partials == nullptr) {
         void* p = nullptr;
-        if (cudaMalloc(&p, (size_t)ctx->ntiles * sizeof(double)) != cudaSuccess) {
+        if (cudaMalloc(&p, (size_t)consensus_blocks((uint32_t)ctx->N) * sizeof(double)) != cudaSuccess) {
             cudaGetLastError();
             return SAPS_ERR_NOMEM;
         }
         ctx->partials = static_cast<double*>(p);
     }
-    return launch_consensus(x, (size_t)ctx->ld, (uint32_t)ctx->N, ctx->n, ctx->ntiles, ctx->partials, out,
+    return launch_consensus(x, (size_t)ctx->ld, (uint32_t)ctx->N, ctx->n, ctx->partials, out,
                             (cudaStream_t)stream) == cudaSuccess
                ? SAPS_OK
                : SAPS_ERR_CUDA;
@@ -479,7 +495,7 @@ int ensure_emit_memory(saps_ctx* ctx)
 {
     if (ctx->emit_mem != nullptr) return SAPS_OK;
     void* p = nullptr;
-    if (cudaMalloc(&p, (size_t)3 * ctx->ntiles * sizeof(uint32_t)) != cudaSuccess) {
+    if (cudaMalloc(&p, ((size_t)2 * ctx->ntiles + (size_t)3 * ctx->ngroups) * sizeof(uint32_t)) != cudaSuccess) {
         cudaGetLastError();
         return SAPS_ERR_NOMEM;
     }
@@ -487,10 +503,10 @@ int ensure_emit_memory(saps_ctx* ctx)
     return SAPS_OK;
 }
 
-// Everything the fused kernel needs to emit round t's wire buffer, enqueued on `stream`:
-// the per-tile counts of round t (taken from the previous call's run-ahead when they are
-// there, counted now otherwise), their prefix, the total.  Fills the emission fields of `a`
-// and arranges for the kernel to count round t+1 ahead.
+// Everything the fused kernel needs to emit round t's wire buffer: the per-tile and per-group
+// counts of round t (taken from the previous call's run-ahead when they are there, counted now
+// on `stream` otherwise).  Fills the emission fields of `a` and arranges for the kernel to count
+// round t+1 ahead.
 int prepare_emission(saps_ctx* ctx, uint64_t t, double keep_frac, uint32_t cap, uint32_t* out_idx,
                      uint32_t* out_count, float* out_vals, cudaStream_t stream, RoundArgs* a)
 {
@@ -498,32 +514,47 @@ int prepare_emission(saps_ctx* ctx, uint64_t t, double keep_frac, uint32_t cap, 
     if (rc != SAPS_OK) return rc;
     rc = ensure_emit_memory(ctx);
     if (rc != SAPS_OK) return rc;
-    const uint32_t nt = ctx->ntiles;
+    const uint32_t nt = ctx->ntiles, ng = ctx->ngroups;
     const uint64_t thr = threshold64(keep_frac);
     uint32_t* cnt_now = ctx->emit_mem + (size_t)ctx->emit_cur * nt;
     uint32_t* cnt_next = ctx->emit_mem + (size_t)(ctx->emit_cur ^ 1) * nt;
-    uint32_t* excl = ctx->emit_mem + (size_t)2 * nt;
+    uint32_t* groups = ctx->emit_mem + (size_t)2 * nt;
+    uint32_t* grp_now = groups + (size_t)ctx->group_cur * ng;
+    uint32_t* grp_next = groups + (size_t)((ctx->group_cur + 1) % 3) * ng;
+    uint32_t* grp_clear = groups + (size_t)((ctx->group_cur + 2) % 3) * ng;
     const bool have = ctx->ahead_valid && ctx->ahead_t == t && ctx->ahead_thr == thr &&
                       ctx->ahead_col_offset == (uint32_t)ctx->col_offset;
     ctx->ahead_valid = false;
-    if (!have && launch_mask_count((uint32_t)ctx->N, (uint32_t)ctx->col_offset, make_key(ctx->seed, t, keep_frac), nt,
-                                   cnt_now, stream) != cudaSuccess)
-        return SAPS_ERR_CUDA;
-    if (launch_tile_scan(cnt_now, nt, excl, out_count, cap, static_cast<int*>(ctx->scratch), stream) != cudaSuccess)
-        return SAPS_ERR_CUDA;
+    if (!have) {
+        // nothing usable from the previous call: clear all group sums, count this round's mask
+        if (cudaMemsetAsync(groups, 0, (size_t)3 * ng * sizeof(uint32_t), stream) != cudaSuccess ||
+            launch_mask_count((uint32_t)ctx->N, (uint32_t)ctx->col_offset, make_key(ctx->seed, t, keep_frac), nt,
+                              cnt_now, grp_now, ctx->group_shift, stream) != cudaSuccess) {
+            cudaGetLastError();
+            return SAPS_ERR_CUDA;
+        }
+    }
     a->out_vals = out_vals;
     a->cap = cap;
-    a->tile_excl = excl;
+    a->tile_cnt = cnt_now;
+    a->group_cnt = grp_now;
     a->out_idx = out_idx;
+    a->out_count = out_count;
+    a->status = static_cast<int*>(ctx->scratch);
     a->next_cnt = nullptr;
+    a->next_group_cnt = nullptr;
+    a->clear_group_cnt = nullptr;
     if (ctx->run_ahead && t + 1 != 0) {
         a->next_cnt = cnt_next;
+        a->next_group_cnt = grp_next;
+        a->clear_group_cnt = grp_clear;
         a->next_key = make_key(ctx->seed, t + 1, keep_frac);
         ctx->ahead_valid = true;   // true once the kernel the caller enqueues next has run
         ctx->ahead_t = t + 1;
         ctx->ahead_thr = thr;
         ctx->ahead_col_offset = (uint32_t)ctx->col_offset;
         ctx->emit_cur ^= 1;
+        ctx->group_cur = (ctx->group_cur + 1) % 3;
     }
     return SAPS_OK;
 }
@@ -541,12 +572,12 @@ int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, const int
     if (rc != SAPS_OK) return rc;
     const RoundKey key = make_key(ctx->seed, t, keep_frac);
     const uint32_t cap = (uint32_t)saps_pack_capacity(ctx, keep_frac);
-    // pass 1 touches no model data: kept columns per tile -> prefixes and count
+    // the kept columns per tile come from the previous call's kernel, or are counted now
     const RowGroups rg = make_groups(ctx->n, pairs, true);
     RoundArgs a = round_args(ctx, x, g, lr, rg, key);
     rc = prepare_emission(ctx, t, keep_frac, cap, out_idx, out_count, out_vals, (cudaStream_t)stream, &a);
     if (rc != SAPS_OK) return rc;
-    // pass 2: the fused round writes the kept columns and each worker's kept values at their ranks
+    // the fused round writes the kept columns and each worker's kept values at their ranks
     rc = timed_round(ctx, a, true, (cudaStream_t)stream);
     if (rc != SAPS_OK) ctx->ahead_valid = false;
     return rc;
@@ -720,8 +751,8 @@ int ensure_lanes(saps_ctx* ctx)
 // and computed on one of a few lane streams (round-robin); its result is copied out on a
 // stream of its own, so that a lane can start its next copy-in without waiting for its last
 // copy-out: the two copy directions and the kernels overlap, and the copy-in queue never
-// runs dry.  With a wire buffer, the mask scan (which touches no model data) runs first on
-// lane 0 and the other lanes wait for its tile prefixes.
+// runs dry.  With a wire buffer whose per-tile counts are not there yet, the counting kernel
+// (which touches no model data) runs first on lane 0 and the other lanes wait for it.
 int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr, const int32_t* pairs,
                     uint64_t t, double keep_frac, float* d_x, float* d_g, const HostPack* pack)
 {
@@ -747,7 +778,7 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
     bool failed = false;
     RoundArgs emit_args = round_args(ctx, d_x, g_host != nullptr ? d_g : nullptr, lr, rg, key, ld_dev);
     if (emit) {
-        // the mask scan touches no model data: it runs first on lane 0, the other lanes wait for it
+        // a counting kernel, if one was needed, runs on lane 0: the other lanes wait for it
         rc = prepare_emission(ctx, t, keep_frac, cap, pack->idx_host != nullptr ? pack->d_idx : nullptr,
                               pack->d_count, pack->d_vals, ctx->lane_stream[0], &emit_args);
         if (rc != SAPS_OK) return rc;
