@@ -197,25 +197,36 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
     }
 }
 
-// Kept columns of every tile under one round's mask (no model data): one warp per tile.
+// Kept columns of every tile under one round's mask (no model data): one block per tile, and
+// the sums over groups of 2^group_shift tiles (group_cnt must be zero before).
 __global__ void __launch_bounds__(kThreads) mask_count_kernel(uint32_t N, uint32_t col_offset, RoundKey key,
-                                                             uint32_t ntiles, uint32_t* tile_cnt, uint32_t* group_cnt,
+                                                             uint32_t* tile_cnt, uint32_t* group_cnt,
                                                              uint32_t group_shift)
 {
-    const int lane = threadIdx.x & 31;
-    const uint32_t tile = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
-    if (tile >= ntiles) return;
-    const uint64_t col0 = (uint64_t)tile * kTileCols;
+    constexpr int kSteps = kTileCols / kThreads;
+    __shared__ uint32_t s_warp_cnt[kThreads / 32];
+    const uint32_t tile = blockIdx.x;
+    const uint32_t col0 = tile * (uint32_t)kTileCols;   // N < 2^32: no wrap
+    const uint32_t rem = N - col0;
+    const uint32_t hash0 = col_offset + col0 + threadIdx.x;
     uint32_t cnt = 0;
-#pragma unroll 8
-    for (int s = 0; s < kTileCols / 32; ++s) {
-        const uint64_t k = col0 + s * 32 + lane;
-        cnt += ((k < N) && column_kept(col_offset + (uint32_t)k, key)) ? 1u : 0u;
+    if (rem >= (uint32_t)kTileCols) {
+#pragma unroll
+        for (int s = 0; s < kSteps; ++s) cnt += column_kept(hash0 + s * kThreads, key) ? 1u : 0u;
+    } else {
+#pragma unroll
+        for (int s = 0; s < kSteps; ++s)
+            cnt += (threadIdx.x + s * kThreads < rem && column_kept(hash0 + s * kThreads, key)) ? 1u : 0u;
     }
-    cnt = warp_sum(cnt);
-    if (lane == 0) {
-        tile_cnt[tile] = cnt;
-        atomicAdd(group_cnt + (tile >> group_shift), cnt);
+    cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+    if ((threadIdx.x & 31) == 0) s_warp_cnt[threadIdx.x >> 5] = cnt;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t total = 0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) total += s_warp_cnt[w];
+        tile_cnt[tile] = total;
+        atomicAdd(group_cnt + (tile >> group_shift), total);
     }
 }
 
@@ -460,9 +471,7 @@ cudaError_t launch_pack_static(PackArgs a, uint32_t ntiles, int* out_status, cud
 cudaError_t launch_mask_count(uint32_t N, uint32_t col_offset, RoundKey key, uint32_t ntiles, uint32_t* tile_cnt,
                               uint32_t* group_cnt, uint32_t group_shift, cudaStream_t stream)
 {
-    const uint32_t per_block = kThreads / 32;
-    mask_count_kernel<<<(ntiles + per_block - 1) / per_block, kThreads, 0, stream>>>(N, col_offset, key, ntiles,
-                                                                                    tile_cnt, group_cnt, group_shift);
+    mask_count_kernel<<<ntiles, kThreads, 0, stream>>>(N, col_offset, key, tile_cnt, group_cnt, group_shift);
     return cudaGetLastError();
 }
 

@@ -23,10 +23,23 @@ namespace {
 class BlossomMatcher {
 public:
     BlossomMatcher(int n, const std::vector<uint8_t>& adj)
-        : n_(n), adj_(adj), mate_(n, -1), up_(n), base_(n), seen_(n), in_blossom_(n), fifo_(n) {}
+        : n_(n), adj_(adj), mate_(n, -1), up_(n), base_(n), seen_(n), in_blossom_(n), on_path_(n), fifo_(n) {}
 
     const std::vector<int>& solve()
     {
+        // start from a greedy matching (first free neighbour of every free vertex): on the dense
+        // graphs of this rule it is already close to maximum, and only the few vertices it
+        // leaves free need a search for an augmenting path
+        for (int v = 0; v < n_; ++v) {
+            if (mate_[v] != -1) continue;
+            for (int w = 0; w < n_; ++w) {
+                if (w != v && mate_[w] == -1 && edge(v, w)) {
+                    mate_[v] = w;
+                    mate_[w] = v;
+                    break;
+                }
+            }
+        }
         for (int v = 0; v < n_; ++v) {
             if (mate_[v] != -1) continue;
             const int leaf = grow_tree(v);
@@ -48,16 +61,16 @@ private:
     // first common blossom base on the two root paths
     int common_base(int a, int b)
     {
-        std::vector<char> on_path(n_, 0);
+        std::fill(on_path_.begin(), on_path_.end(), 0);
         for (int v = a;;) {
             v = base_[v];
-            on_path[v] = 1;
+            on_path_[v] = 1;
             if (mate_[v] == -1) break;
             v = up_[mate_[v]];
         }
         for (int v = b;;) {
             v = base_[v];
-            if (on_path[v]) return v;
+            if (on_path_[v]) return v;
             v = up_[mate_[v]];
         }
     }
@@ -116,7 +129,7 @@ private:
     int n_;
     const std::vector<uint8_t>& adj_;
     std::vector<int> mate_, up_, base_;
-    std::vector<char> seen_, in_blossom_;
+    std::vector<char> seen_, in_blossom_, on_path_;
     std::vector<int> fifo_;
 };
 
@@ -239,11 +252,18 @@ int select_peers(SelectState& st, const double* bandwidth, uint64_t t, int32_t* 
         b_thres = bottleneck_threshold(n, B);
     } else if (st.b_thres_default) {
         std::vector<double> links;
+        links.reserve((size_t)n * (n - 1) / 2);
         for (int i = 0; i < n; ++i)
             for (int j = i + 1; j < n; ++j) links.push_back(B[(size_t)i * n + j]);
-        std::sort(links.begin(), links.end());
+        // median without a full sort: the upper middle element, then the largest below it
         const size_t m = links.size();
-        b_thres = m == 0 ? 0.0 : (m % 2 ? links[m / 2] : 0.5 * (links[m / 2 - 1] + links[m / 2]));
+        if (m == 0) {
+            b_thres = 0.0;
+        } else {
+            std::nth_element(links.begin(), links.begin() + m / 2, links.end());
+            const double upper = links[m / 2];
+            b_thres = m % 2 ? upper : 0.5 * (*std::max_element(links.begin(), links.begin() + m / 2) + upper);
+        }
     }
     int t_thres = st.t_thres;
     if (t_thres == 0) {
