@@ -378,27 +378,33 @@ def run_ours(args):
     # the other entry points of the path, each timed alone on the same resident inputs (context
     # only): a pause lets the power state left by the previous loop settle, and the clocks are
     # sampled while each one runs
-    def timed(fn, reps=20):
+    def timed(fn, min_ms=400.0):
         time.sleep(1.0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         for i in range(3):
             fn(t + i)
-        torch.cuda.synchronize()
-        sampler = ClockSampler(smi_id)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        for i in range(reps):
+        for i in range(10):
             fn(t + 3 + i)
         e1.record(stream)
         torch.cuda.synchronize()
+        reps = int(max(20, min(5000, min_ms / max(e0.elapsed_time(e1) / 10, 1e-3))))
+        sampler = ClockSampler(smi_id)
+        time.sleep(0.3)
+        e0.record(stream)
+        for i in range(reps):
+            fn(t + 13 + i)
+        e1.record(stream)
+        torch.cuda.synchronize()
         c = sampler.stop()
-        return e0.elapsed_time(e1) / reps, {"sm_mhz": c["sm_mhz"], "reasons": c["reasons"]}
+        return e0.elapsed_time(e1) / reps, {"sm_mhz": c["sm_mhz"], "reasons": c["reasons"], "launches": reps}
 
     pairs_fixed = sb.saps_select_peers(ctx, B, t, n)
     t += 1
-    ms_round, ck_round = timed(lambda tt: sb.saps_round(ctx, x, g, w.lr, pairs_fixed, tt, p, stream), reps=40)
-    ms_pack, ck_pack = timed(lambda tt: sb.saps_pack(ctx, x, tt, p, vals, idx, count, stream), reps=200)
+    ms_round, ck_round = timed(lambda tt: sb.saps_round(ctx, x, g, w.lr, pairs_fixed, tt, p, stream))
+    ms_pack, ck_pack = timed(lambda tt: sb.saps_pack(ctx, x, tt, p, vals, idx, count, stream))
     dist_out = torch.zeros(1, dtype=torch.float64, device="cuda")
-    ms_dist, ck_dist = timed(lambda tt: sb.saps_consensus_distance(ctx, x, dist_out, stream), reps=100)
+    ms_dist, ck_dist = timed(lambda tt: sb.saps_consensus_distance(ctx, x, dist_out, stream))
     result["other_entry_points"] = {
         "saps_round": {"ms": ms_round, "algorithmic_gbs": bytes_round / (ms_round * 1e-3) / 1e9,
                        "frac_of_measured_peak": bytes_round / (ms_round * 1e-3) / 1e9 / peak, "clocks": ck_round},
@@ -407,7 +413,7 @@ def run_ours(args):
                                     "frac_of_measured_peak": 4.0 * n * N / (ms_dist * 1e-3) / 1e9 / peak,
                                     "clocks": ck_dist},
     }
-    t += 300
+    t += 6000
 
     if rank == 0 and world == 1 and not args.no_small_loop:
         result["resnet20_scheduler_loop"] = measure_small_loop(sb, synth, stream, peak)

@@ -39,33 +39,32 @@ _lib = None
 
 def _bind(lib):
     """Declare the C signatures on a loaded oracle library."""
-    if True:
-        u32, u64, i32 = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int
-        vp, dbl, f32 = ctypes.c_void_p, ctypes.c_double, ctypes.c_float
-        lib.orc_mix.restype = u32
-        lib.orc_mix.argtypes = [u32]
-        lib.orc_round_key.restype = None
-        lib.orc_round_key.argtypes = [u64, u64, ctypes.POINTER(u32), ctypes.POINTER(u32)]
-        lib.orc_hash.restype = u32
-        lib.orc_hash.argtypes = [u32, u32, u32]
-        lib.orc_threshold.restype = u64
-        lib.orc_threshold.argtypes = [dbl]
-        lib.orc_mask.restype = None
-        lib.orc_mask.argtypes = [u64, u64, dbl, u64, vp]
-        lib.orc_sgd.restype = None
-        lib.orc_sgd.argtypes = [i32, u64, vp, vp, f32]
-        lib.orc_pack.restype = u64
-        lib.orc_pack.argtypes = [i32, u64, vp, vp, u64, vp, vp]
-        lib.orc_pair_average.restype = None
-        lib.orc_pair_average.argtypes = [i32, u64, vp, vp, vp]
-        lib.orc_round.restype = None
-        lib.orc_round.argtypes = [i32, u64, vp, vp, f32, vp, u64, u64, dbl, vp]
-        lib.orc_round_eq7.restype = None
-        lib.orc_round_eq7.argtypes = [i32, u64, vp, vp, f32, vp, u64, u64, dbl, vp]
-        lib.orc_unpack_avg.restype = None
-        lib.orc_unpack_avg.argtypes = [i32, u64, vp, vp, u64, vp, u64]
-        lib.orc_consensus_distance.restype = dbl
-        lib.orc_consensus_distance.argtypes = [i32, u64, vp]
+    u32, u64, i32 = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int
+    vp, dbl, f32 = ctypes.c_void_p, ctypes.c_double, ctypes.c_float
+    lib.orc_mix.restype = u32
+    lib.orc_mix.argtypes = [u32]
+    lib.orc_round_key.restype = None
+    lib.orc_round_key.argtypes = [u64, u64, ctypes.POINTER(u32), ctypes.POINTER(u32)]
+    lib.orc_hash.restype = u32
+    lib.orc_hash.argtypes = [u32, u32, u32]
+    lib.orc_threshold.restype = u64
+    lib.orc_threshold.argtypes = [dbl]
+    lib.orc_mask.restype = None
+    lib.orc_mask.argtypes = [u64, u64, dbl, u64, vp]
+    lib.orc_sgd.restype = None
+    lib.orc_sgd.argtypes = [i32, u64, vp, vp, f32]
+    lib.orc_pack.restype = u64
+    lib.orc_pack.argtypes = [i32, u64, vp, vp, u64, vp, vp]
+    lib.orc_pair_average.restype = None
+    lib.orc_pair_average.argtypes = [i32, u64, vp, vp, vp]
+    lib.orc_round.restype = None
+    lib.orc_round.argtypes = [i32, u64, vp, vp, f32, vp, u64, u64, dbl, vp]
+    lib.orc_round_eq7.restype = None
+    lib.orc_round_eq7.argtypes = [i32, u64, vp, vp, f32, vp, u64, u64, dbl, vp]
+    lib.orc_unpack_avg.restype = None
+    lib.orc_unpack_avg.argtypes = [i32, u64, vp, vp, u64, vp, u64]
+    lib.orc_consensus_distance.restype = dbl
+    lib.orc_consensus_distance.argtypes = [i32, u64, vp]
     return lib
 
 

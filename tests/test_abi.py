@@ -88,10 +88,17 @@ def test_round_rejects_bad_arguments_before_any_launch():
     assert sb._lib.saps_unpack_avg(ctx, fake, None, fake, fake, 0.5, None, None) == sb.SAPS_ERR_INVALID
     assert sb._lib.saps_unpack_avg(ctx, fake, fake, fake, fake, 0.5, sb._pairs([1, 2, 0, 3]), None) == sb.SAPS_ERR_PAIRS
     assert sb._lib.saps_consensus_distance(ctx, fake, None, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_set_host_pipeline(ctx, 0, 7) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_set_host_pipeline(ctx, 0, -1) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_set_host_pipeline(None, 0, 2) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_set_host_pipeline(ctx, 1 << 40, 6) == sb.SAPS_OK
+    assert sb._lib.saps_set_host_pipeline(ctx, 0, 0) == sb.SAPS_OK          # 0 = leave as it is
+    assert sb._lib.saps_round_host(ctx, fake, fake, 0.1, sb._pairs(good), 1, 0.5, None, fake) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_round_host(ctx, fake, fake, 0.1, sb._pairs(good), 1, 0.5, fake, None) == sb.SAPS_ERR_INVALID
     assert sb._lib.saps_set_column_offset(ctx, (1 << 32) - 50) == sb.SAPS_ERR_INVALID
     assert sb._lib.saps_set_column_offset(ctx, (1 << 32) - 100) == sb.SAPS_OK
     sb.saps_destroy(ctx)
-    for code in range(-6, 1):
+    for code in range(-7, 1):
         assert sb.saps_strerror(code) not in ("", "unknown status")
     assert sb.saps_strerror(-99) == "unknown status"
 
