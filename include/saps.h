@@ -135,7 +135,11 @@ SAPS_API int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, 
  * Results are identical either way; enabled = 0 switches the run-ahead off.
  * The counts are kept in the context and read by the next call's kernels, so consecutive
  * emitting calls on one context must run on one stream or be ordered by events (the general
- * rule above that calls on one context must not overlap covers it). */
+ * rule above that calls on one context must not overlap covers it).  To capture a sequence of
+ * emitting calls in a CUDA graph, call saps_set_run_ahead(ctx, 1) right before the capture: that
+ * forgets counts taken by earlier kernels, so the first captured round counts its own mask inside
+ * the graph and every replay is self-contained (make the context's first use before, outside
+ * the capture, since it allocates). */
 SAPS_API int saps_set_run_ahead(saps_ctx* ctx, int enabled);
 
 /* Order of the two halves of the update.

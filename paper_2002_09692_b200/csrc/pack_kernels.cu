@@ -251,7 +251,10 @@ __global__ void __launch_bounds__(kThreads) unpack_avg_kernel(const UnpackArgs a
     const uint32_t k = __ldg(a.idx + r) - a.col_offset;
     if (k >= a.N) return;  // an index list of another shard: stay in bounds
     float* p = a.x + (size_t)blockIdx.y * a.ld + k;
-    *p = __fmul_rn(0.5f, __fadd_rn(*p, __ldg(a.recv + (size_t)src * a.cap + r)));
+    // an isolated value of a row: ask the L2 for 64 bytes, not for the whole 128-byte line
+    float own;
+    asm volatile("ld.global.L2::64B.f32 %0, [%1];" : "=f"(own) : "l"(p) : "memory");
+    *p = __fmul_rn(0.5f, __fadd_rn(own, __ldg(a.recv + (size_t)src * a.cap + r)));
 }
 
 // Consensus distance, one block per kConsensusCols columns (half a column tile: blocks this

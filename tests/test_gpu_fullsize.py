@@ -110,6 +110,41 @@ def test_vgg16_consecutive_rounds_every_element(sb):
     assert float(dx[:, N:].abs().max()) == 0.0
 
 
+def test_vgg16_host_pipeline_every_element(sb):
+    # The end-to-end entry point at the size and in the configuration bench.py times it: pinned
+    # host matrices in, 15 column chunks over three lanes, model and wire buffer out; two
+    # consecutive rounds (the second one uses counts taken ahead by the first one's chunk kernels),
+    # every element against the oracle.
+    torch = torch_cuda()
+    w = synth.WORKLOADS["vgg16"]
+    n, N, ld, p = w.n, w.N, round_up(w.N, 32), 0.01
+    x, g = synth.model_and_grad(w)
+    B = synth.bandwidth_matrix(n, *w.bw_range, seed=w.seed)
+    hx = torch.from_numpy(x.copy()).pin_memory()
+    hg = torch.from_numpy(g).pin_memory()
+    d_x = torch.zeros(n, ld, dtype=torch.float32, device="cuda")
+    d_g = torch.zeros(n, ld, dtype=torch.float32, device="cuda")
+    ctx = sb.saps_create_ld(n, N, ld, w.seed)
+    cap = sb.saps_pack_capacity(ctx, p)
+    hv = torch.zeros(n, cap, dtype=torch.float32).pin_memory()
+    hi = torch.zeros(cap, dtype=torch.int32).pin_memory()
+    hc = torch.zeros(1, dtype=torch.int32).pin_memory()
+    d_v = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
+    d_i = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    d_c = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for t in (1, 2):
+        pairs = sb.saps_select_peers(ctx, B, t, n)
+        sb.saps_round_pack_host(ctx, hx, hg, w.lr, pairs, t, p, d_x, d_g, hv, hi, hc, d_v, d_i, d_c)
+        assert sb.saps_status(ctx) == 0
+        wv, wi, wc = _oracle_round_with_pack(x, g, w, pairs, t, p, cap)
+        assert int(hc[0]) == wc
+        assert (hi.numpy().view(np.uint32)[:wc] == wi[:wc]).all()
+        assert_bits_equal(hv.numpy()[:, :wc], wv[:, :wc], f"host wire buffer, round {t}")
+        assert_bits_equal(hx.numpy(), x, f"host model after round {t}")
+    assert float(d_x[:, N:].abs().max()) == 0.0 and float(d_g[:, N:].abs().max()) == 0.0
+    sb.saps_destroy(ctx)
+
+
 def _sampled_rounds(sb, torch, w, p, pairs_of_round, rows_of_round, golden=None):
     """Bench-style consecutive rounds t = 1, 2, ... on one context (fixed keep_frac, so every
     round after the first uses the counts the previous kernel took ahead) on device-drawn

@@ -340,3 +340,56 @@ def test_run_rounds_pack_emits_every_round(sb):
                                       None, None)
     assert rc == sb.SAPS_ERR_INVALID
     sb.saps_destroy(ctx)
+
+
+def test_scheduler_loop_captured_in_a_cuda_graph_and_replayed(sb):
+    # Every device operation of the library is enqueued on the caller's stream and, after the
+    # first use of a context, nothing is allocated: a round loop can be captured in a CUDA graph.
+    # saps_set_run_ahead just before the capture makes the captured sequence self-contained (its
+    # first round counts its own mask inside the graph instead of relying on a kernel that ran
+    # before the capture).  Replaying the graph repeats the same rounds t = 1..T on the model as
+    # it is then; both executions are checked against the oracle.
+    torch = torch_cuda()
+    w = synth.WORKLOADS["resnet20"]
+    T, p = 10, w.keep_fracs[0]
+    x, g = synth.model_and_grad(w)
+    ld = round_up(w.N, 32)
+    dx, dg = DeviceMatrix(x, ld), DeviceMatrix(g, ld)
+    rng = synth.matching_rng(5)
+    pairs_list = np.stack([synth.random_perfect_matching(w.n, rng) for _ in range(T)]).astype(np.int32)
+    ctx = sb.saps_create_ld(w.n, w.N, ld, w.seed)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.zeros(w.n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    counts = torch.zeros(T, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    # first use outside the capture: the context allocates its scratch here
+    scratch_x = dx.view.clone()
+    with torch.cuda.stream(side):
+        sb.saps_run_rounds_pack(ctx, scratch_x, dg.ptr, w.lr, 1, 2, p, vals, idx, counts, pairs_list=pairs_list[:2],
+                                stream=side)
+    side.synchronize()
+    assert sb.saps_status(ctx, side) == 0
+    sb.saps_set_run_ahead(ctx, True)                      # forget counts taken ahead by the warm-up
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        sb.saps_run_rounds_pack(ctx, dx.ptr, dg.ptr, w.lr, 1, T, p, vals, idx, counts, pairs_list=pairs_list,
+                                stream=torch.cuda.current_stream())
+    want = x.copy()
+    for replay in range(2):
+        graph.replay()
+        torch.cuda.synchronize()
+        assert sb.saps_status(ctx) == 0
+        for t in range(1, T + 1):
+            oracle.sgd(want, g, w.lr)
+            m = oracle.mask(w.seed, t, p, w.N)
+            assert int(counts[t - 1]) == int(m.sum())
+            if t == T:
+                wv, wi, wc = oracle.pack(want, m, cap)
+            oracle.pair_average(want, pairs_list[t - 1], m)
+        assert (idx.cpu().numpy().view(np.uint32)[:wc] == wi[:wc]).all()
+        assert_bits_equal(vals.cpu().numpy()[:, :wc], wv[:, :wc], f"wire buffer after replay {replay}")
+        assert_bits_equal(dx.host(), want, f"model after replay {replay}")
+    assert dx.canaries_intact()
+    del graph
+    sb.saps_destroy(ctx)
