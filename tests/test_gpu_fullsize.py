@@ -222,7 +222,7 @@ def _history_cone(pairs_of_round, last_rows):
 def test_resnet50_keep_frac_sweep_sampled_rows(sb):
     # uniformly random perfect matchings; three consecutive rounds per keep_frac on one context;
     # the oracle follows workers 0 and 17 and everyone whose values reach them (at most 16 rows
-    # in round 1, 8 in round 2, 4 in round 3)
+    # at t = 1, 8 at t = 2, 4 at t = 3)
     torch = torch_cuda()
     w = synth.WORKLOADS["resnet50"]
     rng = synth.matching_rng(w.seed)
@@ -235,7 +235,7 @@ def test_resnet50_keep_frac_sweep_sampled_rows(sb):
 
 def test_gpt2s_sampled_rows(sb):
     # adaptive peer selection (Algorithm 3) for three consecutive rounds; the oracle follows
-    # worker 5 and everyone whose values reach it (8 rows in round 1, 4 in round 2, 2 in round 3)
+    # worker 5 and everyone whose values reach it (8 rows at t = 1, 4 at t = 2, 2 at t = 3)
     torch = torch_cuda()
     w = synth.WORKLOADS["gpt2s"]
     B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
