@@ -69,7 +69,7 @@ __device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t v, int lane)
 // GOSSIP_FIRST selects the order of Eq. 7 (average the current models, then subtract the
 // gradient step) instead of Algorithm 2's (SGD step first, then average).
 template <int VEC, bool HAS_G, bool EMIT, bool GOSSIP_FIRST>
-__global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
+__global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const RoundArgs a)
 {
     constexpr int U = kTileCols / (kThreads * VEC);
     constexpr int kWarps = kThreads / 32;
@@ -141,35 +141,42 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
     uint32_t total = 0;     // EMIT only: kept columns in the vector part of the tile
     uint32_t excl = 0;      // EMIT only: kept columns in all earlier tiles
     if constexpr (EMIT) {
-        __shared__ uint32_t s_warp[U][kWarps];
+        // Two counts travel in one word (16 bits each: a tile keeps at most 2048 columns), so one
+        // warp scan and one pass over the warps' totals serve two of the thread's vectors.
+        static_assert(U % 2 == 0, "vectors are ranked two at a time");
+        constexpr int P = U / 2;
+        __shared__ uint32_t s_warp[P][kWarps];
         __shared__ uint32_t s_excl[32];
         const int lane = tid & 31, warp = tid >> 5;
         {
             const uint32_t e = __reduce_add_sync(0xFFFFFFFFu, excl_part);
             if (lane == 0) s_excl[warp] = e;
         }
-        uint32_t within[U];
+        uint32_t within[P];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t c = __popc(bits[u]);
+        for (int j = 0; j < P; ++j) {
+            const uint32_t c = __popc(bits[2 * j]) | (__popc(bits[2 * j + 1]) << 16);
             const uint32_t inc = warp_inclusive_sum(c, lane);
-            within[u] = inc - c;
-            if (lane == 31) s_warp[u][warp] = inc;
+            within[j] = inc - c;
+            if (lane == 31) s_warp[j][warp] = inc;
         }
         __syncthreads();
         excl = __reduce_add_sync(0xFFFFFFFFu, lane < kWarps ? s_excl[lane] : 0u);
         uint32_t running = excl;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
+        for (int j = 0; j < P; ++j) {
             uint32_t before = 0, all = 0;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) {
-                const uint32_t s = s_warp[u][w];
+                const uint32_t s = s_warp[j][w];
                 before += (w < warp) ? s : 0u;
                 all += s;
             }
-            rank[u] = running + before + within[u];
-            running += all;
+            const uint32_t mine = before + within[j];
+            rank[2 * j] = running + (mine & 0xFFFFu);
+            running += all & 0xFFFFu;
+            rank[2 * j + 1] = running + (mine >> 16);
+            running += all >> 16;
         }
         total = running - excl;
         // the list of kept columns is the same for every row group: the first one writes it
@@ -203,8 +210,7 @@ __global__ void __launch_bounds__(kThreads) round_kernel(const RoundArgs a)
                 if ((uint32_t)tid < a.N - nfull && col_tile <= nfull && nfull < col_tile + kTileCols)
                     c += column_kept(a.col_offset + nfull + tid, a.next_key) ? 1u : 0u;
             }
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, d);
+            c = __reduce_add_sync(0xFFFFFFFFu, c);
             if (lane == 0) s_next[warp] = c;
             __syncthreads();
             if (tid == 0) {
