@@ -209,24 +209,25 @@ double bottleneck_threshold(int n, const std::vector<double>& B)
 }
 
 // FindConnectedSubgraph: component label per vertex; returns the number of components.
-int label_components(int n, const std::vector<uint8_t>& Q, std::vector<int>& label)
+// n <= 64, so a row of the (symmetric) graph is one 64-bit mask and a component grows by whole
+// rows at a time.
+int label_components(int n, const uint64_t* row, std::vector<int>& label)
 {
     label.assign(n, -1);
+    uint64_t unvisited = n == 64 ? ~0ull : ((1ull << n) - 1);
     int c = 0;
-    std::vector<int> stack;
-    for (int s = 0; s < n; ++s) {
-        if (label[s] != -1) continue;
-        label[s] = c;
-        stack.push_back(s);
-        while (!stack.empty()) {
-            const int v = stack.back();
-            stack.pop_back();
-            for (int w = 0; w < n; ++w)
-                if (Q[(size_t)v * n + w] && label[w] == -1) {
-                    label[w] = c;
-                    stack.push_back(w);
-                }
+    while (unvisited != 0) {
+        const int s = __builtin_ctzll(unvisited);
+        uint64_t comp = 1ull << s, frontier = comp;
+        while (frontier != 0) {
+            const int v = __builtin_ctzll(frontier);
+            frontier &= frontier - 1;
+            const uint64_t fresh = row[v] & ~comp;
+            comp |= fresh;
+            frontier |= fresh;
         }
+        for (uint64_t m = comp; m != 0; m &= m - 1) label[__builtin_ctzll(m)] = c;
+        unvisited &= ~comp;
         ++c;
     }
     return c;
@@ -272,14 +273,18 @@ int select_peers(SelectState& st, const double* bandwidth, uint64_t t, int32_t* 
         t_thres = std::max(2, 2 * lg);
     }
 
-    // IfConnected: recently connected edges, R_ij > t - T_thres
-    std::vector<uint8_t> Q((size_t)n * n, 0);
+    // IfConnected: recently connected edges, R_ij > t - T_thres.  "Never" is far below every
+    // horizon, so the one comparison covers it; an edge counts when either direction is recent.
     const int64_t horizon = (int64_t)t - (int64_t)t_thres;
+    uint64_t Q[kMaxWorkers] = {};
+    for (int i = 0; i < n; ++i) {
+        const int64_t* r = &st.R[(size_t)i * n];
+        uint64_t bits = 0;
+        for (int j = 0; j < n; ++j) bits |= (uint64_t)(r[j] > horizon) << j;
+        Q[i] |= bits & ~(1ull << i);
+    }
     for (int i = 0; i < n; ++i)
-        for (int j = 0; j < n; ++j) {
-            const int64_t r = st.R[(size_t)i * n + j];
-            if (i != j && r != kNever && r > horizon) Q[(size_t)i * n + j] = Q[(size_t)j * n + i] = 1;
-        }
+        for (uint64_t m = Q[i]; m != 0; m &= m - 1) Q[__builtin_ctzll(m)] |= 1ull << i;
     std::vector<int> label;
     const int ncomp = label_components(n, Q, label);
 
