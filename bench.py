@@ -335,9 +335,9 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": dict(workload_config(w, p, world),
-                       gpu_step="saps_select_peers + saps_round_pack (one fused SGD/mask/emit/average kernel per step; "
-                                "it also counts the next round's mask per tile, so no separate scan runs)"),
+        "config": workload_config(w, p, world),
+        "gpu_step": "saps_select_peers + saps_round_pack (one fused SGD/mask/emit/average kernel per step; "
+                    "it also counts the next round's mask per tile, so no separate scan runs)",
         "effective_hbm_gbs": bytes_round * K / (elapsed_ms * 1e-3) / 1e9,
         "frac_of_8tbs": bytes_round * K / (elapsed_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
         "kept_columns": kept,
