@@ -248,6 +248,88 @@ def test_gpt2s_sampled_rows(sb):
     torch.cuda.empty_cache()
 
 
+def _many_rounds_on_column_windows(sb, torch, w, p, T, windows, bandwidth=None, pairs_list=None):
+    """The configured number of rounds at full size in ONE scheduler call (saps_run_rounds_pack),
+    followed on the CPU by the oracle on a few column windows of ALL workers: the mask depends on
+    the column only and the update acts column by column, so a window can be replayed on its own
+    (SGD step, that window of the full-length oracle mask, pair average).  Checked: every round's
+    count against the oracle's mask, the final model on the windows, the last round's index list
+    and the windows' part of the last wire buffer."""
+    n, N, ld = w.n, w.N, round_up(w.N, 32)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(4321 + T)
+    dx = torch.empty(n, ld, dtype=torch.float32, device="cuda").normal_(0.0, w.x_std, generator=gen)
+    dg = torch.empty(n, ld, dtype=torch.float32, device="cuda").normal_(0.0, w.g_std, generator=gen)
+    xs = [np.ascontiguousarray(dx[:, c0:c1].cpu().numpy()) for c0, c1 in windows]
+    gs = [np.ascontiguousarray(dg[:, c0:c1].cpu().numpy()) for c0, c1 in windows]
+    padding = dx[:, N:].clone()
+    ctx = sb.saps_create_ld(n, N, ld, w.seed)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    counts = torch.zeros(T, dtype=torch.int32, device="cuda")
+    log = np.zeros((T, n), dtype=np.int32)
+    sb.saps_run_rounds_pack(ctx, dx, dg, w.lr, 1, T, p, vals, idx, counts, pairs_list=pairs_list,
+                            bandwidth=bandwidth, out_pairs_log=log)
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    sb.saps_destroy(ctx)
+    got_counts = counts.cpu().numpy().view(np.uint32)
+    for t in range(1, T + 1):
+        m = oracle.mask(w.seed, t, p, N)
+        assert int(got_counts[t - 1]) == int(m.sum(dtype=np.int64)), f"count of round {t}"
+        for (c0, c1), xw, gw in zip(windows, xs, gs):
+            oracle.sgd(xw, gw, w.lr)
+            if t == T:
+                kept = np.nonzero(m)[0]
+                c = len(kept)
+                assert (idx[:c].cpu().numpy().view(np.uint32) == kept.astype(np.uint32)).all()
+                lo, hi = np.searchsorted(kept, [c0, c1])
+                assert_bits_equal(vals[:, lo:hi].cpu().numpy(), xw[:, kept[lo:hi] - c0],
+                                  f"last wire buffer, columns [{c0}, {c1})")
+            oracle.pair_average(xw, log[t - 1], np.ascontiguousarray(m[c0:c1]))
+    for (c0, c1), xw in zip(windows, xs):
+        assert_bits_equal(dx[:, c0:c1].cpu().numpy(), xw, f"model after {T} rounds, columns [{c0}, {c1})")
+    assert torch.equal(dx[:, N:], padding)                 # columns beyond N are never written
+    return log
+
+
+def _windows(N):
+    # the first tiles, an unaligned stretch in the middle, and the ragged end of the rows
+    mid = (N // 2) | 1
+    return [(0, 150_000), (mid, mid + 100_001), (N - 150_003, N)]
+
+
+def test_vgg16_fifty_rounds_adaptive_selection(sb):
+    # 50 rounds at each keep_frac with Algorithm 3 choosing the peers, as the workload is specified
+    torch = torch_cuda()
+    w = synth.WORKLOADS["vgg16"]
+    B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
+    for p in w.keep_fracs:
+        log = _many_rounds_on_column_windows(sb, torch, w, p, w.rounds, _windows(w.N), bandwidth=B)
+        assert len({tuple(r) for r in log}) > 25            # the matching keeps changing
+        torch.cuda.empty_cache()
+
+
+def test_resnet50_twenty_rounds_per_keep_frac(sb):
+    # uniformly random perfect matching per round, 20 rounds for each keep_frac of the sweep
+    torch = torch_cuda()
+    w = synth.WORKLOADS["resnet50"]
+    rng = synth.matching_rng(w.seed)
+    for p in w.keep_fracs:
+        pairs_list = np.stack([synth.random_perfect_matching(w.n, rng) for _ in range(w.rounds)]).astype(np.int32)
+        _many_rounds_on_column_windows(sb, torch, w, p, w.rounds, _windows(w.N), pairs_list=pairs_list)
+        torch.cuda.empty_cache()
+
+
+def test_gpt2s_ten_rounds_adaptive_selection(sb):
+    torch = torch_cuda()
+    w = synth.WORKLOADS["gpt2s"]
+    B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
+    _many_rounds_on_column_windows(sb, torch, w, w.keep_fracs[0], w.rounds, _windows(w.N), bandwidth=B)
+    torch.cuda.empty_cache()
+
+
 def test_largest_column_count(sb):
     # N just below 2^32 (the largest the 32-bit column index allows), ragged (N mod 4 = 3),
     # two workers, pure gossip with emission.  Checked against the oracle's hash on sampled and
