@@ -80,15 +80,19 @@ def test_run_rounds_with_learning_rate_schedule(sb):
         assert_bits_equal(dx.host(), want, f"schedule, order {order}")
 
 
-@pytest.mark.parametrize("N,p", [(33, 0.5), (70_001, 0.05), (300_000, 0.01), (4096, 1.0), (5000, 0.0)])
-def test_wire_path_sgd_pack_exchange_unpack(sb, N, p):
-    # SGD-only round -> saps_pack -> (buffers travel) -> saps_unpack_avg  ==  fused saps_round
+@pytest.mark.parametrize("N,p", [(33, 0.5), (70_001, 0.05), (300_000, 0.01), (4096, 1.0), (5000, 0.0),
+                                 (70_001, 0.5), (2043, 1.0)])
+@pytest.mark.parametrize("align", [4, 8, 32])
+def test_wire_path_sgd_pack_exchange_unpack(sb, N, p, align):
+    # SGD-only round -> saps_pack -> (buffers travel) -> saps_unpack_avg  ==  fused saps_round,
+    # for sparse and dense masks (several kept columns per 32-byte sector) and row strides of
+    # every alignment.
     torch = torch_cuda()
     n, lr = 6, 0.05
     pairs = [3, 4, 2, 0, 1, 5]                  # workers 2 and 5 have no peer
     x = synth.gaussian_matrix(n, N, 1.0, 25, 0)
     g = synth.gaussian_matrix(n, N, 0.01, 25, 1)
-    ld = round_up(N, 4)
+    ld = round_up(N, align) + (4 if align == 4 and round_up(N, 4) % 8 == 0 else 0)
     ctx = sb.saps_create_ld(n, N, ld, 25)
     fused, dg = DeviceMatrix(x, ld), DeviceMatrix(g, ld)
     sb.saps_round(ctx, fused.ptr, dg.ptr, lr, pairs, 2, p)
