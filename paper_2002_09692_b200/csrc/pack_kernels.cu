@@ -97,11 +97,13 @@ __device__ __forceinline__ float load_gather(const float* p)
     return v;
 }
 
-template <bool GATHER>
-__global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
+// THREADS = 256, or 128 for very sparse masks (a tile then has fewer values to gather than a
+// large block has threads, and more, smaller blocks hide the look-back's latency better).
+template <bool GATHER, int THREADS>
+__global__ void __launch_bounds__(THREADS) pack_kernel(const PackArgs a)
 {
-    constexpr int kWarps = kThreads / 32;
-    constexpr int kSteps = kTileCols / kThreads;  // ballots per warp
+    constexpr int kWarps = THREADS / 32;
+    constexpr int kSteps = kTileCols / THREADS;  // ballots per warp
     __shared__ uint32_t s_tile, s_excl, s_abort;
     __shared__ uint32_t s_warp_cnt[kWarps];
     __shared__ uint16_t s_kept[kTileCols];        // kept columns as offsets inside the tile
@@ -180,7 +182,7 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
     const uint32_t room = base < a.cap ? a.cap - base : 0u;
     const uint32_t take = total < room ? total : room;
     if (a.out_idx != nullptr)
-        for (uint32_t q = tid; q < take; q += kThreads) a.out_idx[base + q] = a.col_offset + col0 + s_kept[q];
+        for (uint32_t q = tid; q < take; q += THREADS) a.out_idx[base + q] = a.col_offset + col0 + s_kept[q];
 
     // ---- gather: only the kept lanes of x are ever loaded ----
     if constexpr (GATHER) {
@@ -190,7 +192,7 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
         const float* xt = a.x + col0;
         const uint32_t items = (uint32_t)a.n * take;
 #pragma unroll 4
-        for (uint32_t e = tid; e < items; e += kThreads) {
+        for (uint32_t e = tid; e < items; e += THREADS) {
             const uint32_t i = e / take, q = e - i * take;
             a.out_vals[(size_t)i * a.cap + base + q] = load_gather(xt + (size_t)i * a.ld + s_kept[q]);
         }
@@ -421,12 +423,22 @@ cudaError_t launch_consensus(const float* x, size_t ld, uint32_t N, int n, doubl
     return cudaLaunchKernelEx(&cfg, consensus_final_kernel, (const double*)partials, blocks, out);
 }
 
+// Block size by the expected number of values a tile gathers (n workers x kept columns per tile).
+static void launch_pack_kernel(const PackArgs& a, uint32_t ntiles, cudaStream_t stream)
+{
+    const double kept_per_tile = a.key.all ? (double)kTileCols : (double)kTileCols * a.key.thr32 / 4294967296.0;
+    if ((double)a.n * kept_per_tile < 128.0)
+        pack_kernel<true, 128><<<ntiles, 128, 0, stream>>>(a);
+    else
+        pack_kernel<true, kThreads><<<ntiles, kThreads, 0, stream>>>(a);
+}
+
 cudaError_t launch_pack(const PackArgs& a, cudaStream_t stream)
 {
     const uint32_t ntiles = a.scratch.ntiles;
     cudaError_t e = cudaMemsetAsync(a.scratch.ticket, 0, scratch_clear_bytes(ntiles), stream);
     if (e != cudaSuccess) return e;
-    pack_kernel<true><<<ntiles, kThreads, 0, stream>>>(a);
+    launch_pack_kernel(a, ntiles, stream);
     return cudaGetLastError();
 }
 
@@ -463,7 +475,7 @@ cudaError_t launch_pack_static(PackArgs a, uint32_t ntiles, int* out_status, cud
     // the area keeps whatever the previous call left: status, ticket and tile states restart at zero
     e = cudaMemsetAsync(base, 0, 4 + scratch_clear_bytes(ntiles), stream);
     if (e != cudaSuccess) return e;
-    pack_kernel<true><<<ntiles, kThreads, 0, stream>>>(a);
+    launch_pack_kernel(a, ntiles, stream);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (out_status != nullptr)
