@@ -31,6 +31,17 @@ def test_library_exports_every_declared_symbol():
     assert sorted(sb.EXPORTS) == names, "binding and header disagree"
 
 
+def test_header_is_plain_c():
+    # the boundary is a C ABI: the header must compile as C99 without warnings
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    out = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c",
+                          os.path.join(ROOT, "include", "saps.h")], capture_output=True, text=True)
+    assert out.returncode == 0, out.stderr
+
+
 def test_round_key_and_threshold_golden():
     for rec in golden_records("mask_hash.txt"):
         if rec[0] == "key":
