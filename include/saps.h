@@ -154,6 +154,17 @@ SAPS_API int saps_set_run_ahead(saps_ctx* ctx, int enabled);
 #define SAPS_ORDER_GOSSIP_FIRST 1
 SAPS_API int saps_set_update_order(saps_ctx* ctx, int order);
 
+/* How the fused round moves its row pieces when rows allow 128-bit accesses and there is a
+ * gradient.  SAPS_STAGING_BULK: bulk asynchronous copies global -> shared memory (completion on
+ * an mbarrier, bounded wait), results back by bulk copies shared -> global; the fastest form for
+ * models that stream from HBM.  SAPS_STAGING_REGISTERS: vector loads and stores from registers;
+ * the better form for models that stay in L2 and the only one for other row alignments.
+ * SAPS_STAGING_AUTO (default) chooses by the size of the launch.  Results are bit-identical. */
+#define SAPS_STAGING_AUTO      0
+#define SAPS_STAGING_REGISTERS 1
+#define SAPS_STAGING_BULK      2
+SAPS_API int saps_set_staging(saps_ctx* ctx, int staging);
+
 /* ---- pack (Eq. 2; "sends the non-zero elements", Section II-B) -------------------------- */
 
 /* Slots per worker that out_vals / out_idx must hold for this keep_frac:

@@ -63,6 +63,7 @@ _SIGNATURES = {
     "saps_run_rounds": (_i32, [_vp, _vp, _vp, _f32, _u64, _u64, _f64, _vp, _vp, _vp, _vp, _vp]),
     "saps_run_rounds_pack": (_i32, [_vp, _vp, _vp, _f32, _u64, _u64, _f64, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "saps_set_update_order": (_i32, [_vp, _i32]),
+    "saps_set_staging": (_i32, [_vp, _i32]),
     "saps_set_run_ahead": (_i32, [_vp, _i32]),
     "saps_unpack_avg": (_i32, [_vp, _vp, _vp, _vp, _vp, _f64, _vp, _vp]),
     "saps_unpack_avg_rows": (_i32, [_vp, _vp, _vp, _vp, _vp, _f64, _vp, _vp]),
@@ -253,6 +254,13 @@ SAPS_ORDER_GOSSIP_FIRST = 1
 
 def saps_set_update_order(ctx, order: int) -> None:
     _check(_lib.saps_set_update_order(ctx, order), "saps_set_update_order")
+
+
+SAPS_STAGING_AUTO, SAPS_STAGING_REGISTERS, SAPS_STAGING_BULK = 0, 1, 2
+
+
+def saps_set_staging(ctx, staging: int) -> None:
+    _check(_lib.saps_set_staging(ctx, staging), "saps_set_staging")
 
 
 def saps_set_run_ahead(ctx, enabled: bool) -> None:

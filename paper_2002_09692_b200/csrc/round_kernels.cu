@@ -66,11 +66,46 @@ __device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t v, int lane)
     return v;
 }
 
+
+// ---- bulk asynchronous copies (global <-> shared memory, completion on an mbarrier) -------------
+// Used by the 128-bit form of the round with gradients: one thread asks the copy engine for the
+// block's four (or two) row pieces, everybody hashes the mask meanwhile, and the results leave the
+// same way.  Addresses are 16-byte aligned and sizes multiples of 16 bytes by construction (the
+// caller takes this path only for ld % 4 == 0 and 16-byte aligned bases; a tile starts at a
+// multiple of 2048 columns and covers a multiple of 4).  No multicast, no other CTA involved.
+__device__ __forceinline__ uint32_t shared_address(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void bulk_load(float* dst_shared, const float* src_global, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(shared_address(dst_shared)), "l"(src_global), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void bulk_store(float* dst_global, const float* src_shared, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 :: "l"(dst_global), "r"(shared_address(src_shared)), "r"(bytes) : "memory");
+}
+
+// Bounded wait for phase 0 of the barrier (every poll is itself a time-limited hardware wait).
+constexpr uint32_t kBulkPolls = 1u << 20;
+__device__ __forceinline__ bool bulk_wait(uint32_t bar)
+{
+    uint32_t done = 0;
+    for (uint32_t it = 0; it < kBulkPolls && !done; ++it) {
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+                     : "=r"(done) : "r"(bar), "r"(0u) : "memory");
+    }
+    return done != 0;
+}
+
 // GOSSIP_FIRST selects the order of Eq. 7 (average the current models, then subtract the
 // gradient step) instead of Algorithm 2's (SGD step first, then average).
-template <int VEC, bool HAS_G, bool EMIT, bool GOSSIP_FIRST>
+// BULK (VEC = 4 with gradients only): the row pieces travel through shared memory by bulk copies.
+template <int VEC, bool HAS_G, bool EMIT, bool GOSSIP_FIRST, bool BULK>
 __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const RoundArgs a)
 {
+    static_assert(!BULK || (VEC == 4 && HAS_G), "bulk copies serve the 128-bit form with gradients");
     constexpr int U = kTileCols / (kThreads * VEC);
     constexpr int kWarps = kThreads / 32;
     const int tid = threadIdx.x;
@@ -89,6 +124,31 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
     const uint32_t nfull = a.N - a.N % VEC;
     const uint64_t col_tile = (uint64_t)tile * kTileCols;
 
+    // BULK: staging buffers x_a, g_a, x_b, g_b of the tile and the barrier their copies complete on
+    __shared__ __align__(128) float s_stage[BULK ? 4 : 1][BULK ? kTileCols : 4];
+    __shared__ __align__(8) unsigned long long s_bar;
+    uint32_t bulk_bytes = 0;
+    if constexpr (BULK) {
+        const uint32_t bar = shared_address(&s_bar);
+        const uint32_t cols = nfull > col_tile ? (uint32_t)(nfull - col_tile < kTileCols ? nfull - col_tile : kTileCols) : 0u;
+        bulk_bytes = cols * (uint32_t)sizeof(float);
+        if (tid == 0) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar));
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncthreads();
+        if (tid == 0 && bulk_bytes != 0) {
+            const uint32_t pieces = paired ? 4u : 2u;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(pieces * bulk_bytes) : "memory");
+            bulk_load(s_stage[0], xa + col_tile, bulk_bytes, bar);
+            bulk_load(s_stage[1], ga + col_tile, bulk_bytes, bar);
+            if (paired) {
+                bulk_load(s_stage[2], xb + col_tile, bulk_bytes, bar);
+                bulk_load(s_stage[3], gb + col_tile, bulk_bytes, bar);
+            }
+        }
+    }
+
     Chunk<VEC> va[U], vb[U], wa[U], wb[U];
     bool inb[U];
     uint32_t col[U];
@@ -98,7 +158,7 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
         const uint64_t k = col_tile + (uint64_t)(u * kThreads + tid) * VEC;
         inb[u] = k < nfull;
         col[u] = (uint32_t)k;
-        if (inb[u]) {
+        if (!BULK && inb[u]) {
             va[u] = load_stream<VEC>(xa + k);
             if (HAS_G) wa[u] = load_stream<VEC>(ga + k);
             if (paired) {
@@ -127,11 +187,51 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
 #pragma unroll
             for (int c = 0; c < VEC; ++c)
                 bits[u] |= (column_kept(a.col_offset + col[u] + c, a.key) ? 1u : 0u) << c;
-            if (HAS_G && !GOSSIP_FIRST) {
+            if (!BULK && HAS_G && !GOSSIP_FIRST) {
 #pragma unroll
                 for (int c = 0; c < VEC; ++c) {
                     va[u].v[c] = sgd_step(va[u].v[c], wa[u].v[c], a.lr);
                     if (paired) vb[u].v[c] = sgd_step(vb[u].v[c], wb[u].v[c], a.lr);
+                }
+            }
+        }
+    }
+
+    // BULK: the staged pieces have arrived (or, should the bounded wait ever run out, the thread
+    // reads its vectors straight from global memory: same values, and the status word says so)
+    bool staged = false;
+    if constexpr (BULK) {
+        staged = bulk_bytes != 0 && bulk_wait(shared_address(&s_bar));
+        if (bulk_bytes != 0 && !staged && a.status != nullptr) atomicCAS(a.status, 0, -5 /* SAPS_ERR_TIMEOUT */);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (inb[u]) {
+                const int v = (u * kThreads + tid) * VEC;
+                if (staged) {
+                    const float4 p0 = *reinterpret_cast<const float4*>(&s_stage[0][v]);
+                    const float4 p1 = *reinterpret_cast<const float4*>(&s_stage[1][v]);
+                    va[u].v[0] = p0.x; va[u].v[1] = p0.y; va[u].v[2] = p0.z; va[u].v[3] = p0.w;
+                    wa[u].v[0] = p1.x; wa[u].v[1] = p1.y; wa[u].v[2] = p1.z; wa[u].v[3] = p1.w;
+                    if (paired) {
+                        const float4 p2 = *reinterpret_cast<const float4*>(&s_stage[2][v]);
+                        const float4 p3 = *reinterpret_cast<const float4*>(&s_stage[3][v]);
+                        vb[u].v[0] = p2.x; vb[u].v[1] = p2.y; vb[u].v[2] = p2.z; vb[u].v[3] = p2.w;
+                        wb[u].v[0] = p3.x; wb[u].v[1] = p3.y; wb[u].v[2] = p3.z; wb[u].v[3] = p3.w;
+                    }
+                } else {
+                    va[u] = load_stream<VEC>(xa + col[u]);
+                    wa[u] = load_stream<VEC>(ga + col[u]);
+                    if (paired) {
+                        vb[u] = load_stream<VEC>(xb + col[u]);
+                        wb[u] = load_stream<VEC>(gb + col[u]);
+                    }
+                }
+                if (!GOSSIP_FIRST) {
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c) {
+                        va[u].v[c] = sgd_step(va[u].v[c], wa[u].v[c], a.lr);
+                        if (paired) vb[u].v[c] = sgd_step(vb[u].v[c], wb[u].v[c], a.lr);
+                    }
                 }
             }
         }
@@ -261,7 +361,13 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
                         vb[u].v[c] = sgd_step(vb[u].v[c], wb[u].v[c], a.lr);
                     }
                 }
-                if (HAS_G || bits[u]) {
+                if (BULK) {
+                    if (staged) {
+                        const int v = (u * kThreads + tid) * VEC;
+                        *reinterpret_cast<float4*>(&s_stage[0][v]) = make_float4(va[u].v[0], va[u].v[1], va[u].v[2], va[u].v[3]);
+                        *reinterpret_cast<float4*>(&s_stage[2][v]) = make_float4(vb[u].v[0], vb[u].v[1], vb[u].v[2], vb[u].v[3]);
+                    }
+                } else if (HAS_G || bits[u]) {
                     store_stream<VEC>(xa + col[u], va[u]);
                     store_stream<VEC>(xb + col[u], vb[u]);
                 }
@@ -270,8 +376,41 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
 #pragma unroll
                     for (int c = 0; c < VEC; ++c) va[u].v[c] = sgd_step(va[u].v[c], wa[u].v[c], a.lr);
                 }
-                store_stream<VEC>(xa + col[u], va[u]);
+                if (BULK) {
+                    if (staged) {
+                        const int v = (u * kThreads + tid) * VEC;
+                        *reinterpret_cast<float4*>(&s_stage[0][v]) = make_float4(va[u].v[0], va[u].v[1], va[u].v[2], va[u].v[3]);
+                    }
+                } else {
+                    store_stream<VEC>(xa + col[u], va[u]);
+                }
             }
+        }
+    }
+
+    if constexpr (BULK) {
+        // The results leave as two bulk stores when every thread had its inputs staged (so nothing
+        // can still arrive in the buffers); otherwise every thread stores its own registers.
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const bool all_staged = __syncthreads_and(staged || bulk_bytes == 0) != 0;
+        if (all_staged) {
+            if (tid == 0 && bulk_bytes != 0) {
+                bulk_store(xa + col_tile, s_stage[0], bulk_bytes);
+                if (paired) bulk_store(xb + col_tile, s_stage[2], bulk_bytes);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the buffers are free again
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (inb[u]) {
+                    store_stream<VEC>(xa + col[u], va[u]);
+                    if (paired) store_stream<VEC>(xb + col[u], vb[u]);
+                }
+            }
+            // copies that were not seen to complete still target this block's buffers: give them
+            // one more bounded wait before the block ends
+            if (tid == 0) bulk_wait(shared_address(&s_bar));
         }
     }
 
@@ -338,11 +477,29 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
     }
 }
 
+// A launch of fewer blocks than this serves a model that stays in L2, where the two extra block
+// barriers of the staged form cost more than its better use of the memory system gains.
+constexpr uint64_t kBulkMinBlocks = 4096;
+
 template <int VEC, bool HAS_G, bool EMIT, bool GOSSIP_FIRST>
 cudaError_t launch_variant(const RoundArgs& a, cudaStream_t stream)
 {
     dim3 grid(a.tile_count, a.groups.count, 1);
-    round_kernel<VEC, HAS_G, EMIT, GOSSIP_FIRST><<<grid, kThreads, 0, stream>>>(a);
+    if constexpr (VEC == 4 && HAS_G) {
+        // 128-bit accesses with gradients: staged through shared memory by bulk copies (32 KB a
+        // block) for models that stream from HBM
+        const bool bulk = a.staging == 2 || (a.staging == 0 && (uint64_t)a.tile_count * a.groups.count >= kBulkMinBlocks);
+        if (bulk) {
+            auto kernel = round_kernel<VEC, HAS_G, EMIT, GOSSIP_FIRST, true>;
+            // once per process and kernel: let five blocks of 32 KB share an SM
+            static const cudaError_t carve =
+                cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+            if (carve != cudaSuccess) return carve;
+            kernel<<<grid, kThreads, 0, stream>>>(a);
+            return cudaGetLastError();
+        }
+    }
+    round_kernel<VEC, HAS_G, EMIT, GOSSIP_FIRST, false><<<grid, kThreads, 0, stream>>>(a);
     return cudaGetLastError();
 }
 

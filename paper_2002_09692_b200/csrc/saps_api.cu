@@ -19,6 +19,7 @@ struct saps_ctx {
     uint64_t col_offset;    // global index of column 0 when this context holds a column shard
     cudaEvent_t ev_before, ev_after;  // optional: recorded around the round kernel
     int gossip_first;       // update order: 0 Algorithm 2, 1 Eq. 7
+    int staging;            // SAPS_STAGING_*
     uint32_t spin_limit;    // poll budget of the look-back
     uint32_t skip_tile;     // test hook, 0xFFFFFFFF = off
     double* partials;       // device, for the consensus distance: one double per block of columns
@@ -157,6 +158,7 @@ RoundArgs round_args(const saps_ctx* ctx, float* x, const float* g, float lr, co
     a.tile_begin = 0;
     a.tile_count = ctx->ntiles;
     a.gossip_first = ctx->gossip_first;
+    a.staging = ctx->staging;
     a.out_vals = nullptr;
     a.cap = 0;
     a.tile_cnt = nullptr;
@@ -210,6 +212,7 @@ int saps_create_ld(int n, uint64_t N, uint64_t ld, uint64_t seed, saps_ctx** out
     ctx->ntiles = (uint32_t)((N + kTileCols - 1) / kTileCols);
     ctx->cap_override = 0;
     ctx->gossip_first = 0;
+    ctx->staging = SAPS_STAGING_AUTO;
     ctx->spin_limit = kSpinLimit;
     ctx->skip_tile = 0xFFFFFFFFu;
     ctx->partials = nullptr;
@@ -310,6 +313,13 @@ int saps_set_column_offset(saps_ctx* ctx, uint64_t col_offset)
 {
     if (ctx == nullptr || col_offset + ctx->N > (1ull << 32)) return SAPS_ERR_INVALID;
     ctx->col_offset = col_offset;
+    return SAPS_OK;
+}
+
+int saps_set_staging(saps_ctx* ctx, int staging)
+{
+    if (ctx == nullptr || staging < SAPS_STAGING_AUTO || staging > SAPS_STAGING_BULK) return SAPS_ERR_INVALID;
+    ctx->staging = staging;
     return SAPS_OK;
 }
 

@@ -62,3 +62,22 @@ def assert_bits_equal(got: np.ndarray, want: np.ndarray, what: str = ""):
         first = tuple(int(v) for v in bad[0])
         raise AssertionError(f"{what}: {len(bad)} of {g.size} words differ, first at {first}: "
                              f"{got[first]!r} != {want[first]!r}")
+
+
+def force_staging(monkeypatch, mode: str) -> None:
+    """Make every context created through the binding use the given staging of the fused round
+    ("auto" leaves the default).  Small test sizes would otherwise never reach the bulk-copy form,
+    which the library only picks for launches of several thousand blocks."""
+    if mode == "auto":
+        return
+    from paper_2002_09692_b200 import binding
+    value = {"registers": binding.SAPS_STAGING_REGISTERS, "bulk": binding.SAPS_STAGING_BULK}[mode]
+    for name in ("saps_create", "saps_create_ld"):
+        original = getattr(binding, name)
+
+        def wrapped(*args, _original=original):
+            ctx = _original(*args)
+            binding.saps_set_staging(ctx, value)
+            return ctx
+
+        monkeypatch.setattr(binding, name, wrapped)

@@ -10,6 +10,14 @@ from gpu_util import DeviceMatrix, assert_bits_equal, round_up, torch_cuda
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(autouse=True, params=["auto", "bulk"])
+def staging(request, monkeypatch):
+    # every test of this file runs with the default choice of the round's staging and with the
+    # bulk-copy form forced (the default only picks it for launches of several thousand blocks)
+    from gpu_util import force_staging
+    force_staging(monkeypatch, request.param)
+
+
 @pytest.fixture(scope="module")
 def sb():
     torch_cuda()
