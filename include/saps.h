@@ -364,6 +364,14 @@ SAPS_API int saps_set_timing_events(saps_ctx* ctx, void* before, void* after);
  * hanging.  skip_tile = 0xFFFFFFFF switches the hook off.  Nothing faults or traps. */
 SAPS_API int saps_debug_inject(saps_ctx* ctx, uint32_t skip_tile, uint32_t spin_limit);
 
+/* Test hook for the bounded wait of the staged form of the fused round (SAPS_STAGING_BULK):
+ * with give_up != 0 every block treats the wait for its bulk copies as run out.  Its threads
+ * then load their vectors straight from global memory and store their results themselves (same
+ * bits), the block still waits, bounded, for its copies to land before it ends, and the status
+ * word receives SAPS_ERR_TIMEOUT when the context has its scratch (any earlier saps_pack or
+ * emitting call creates it).  Every access stays in bounds; nothing faults, traps or hangs. */
+SAPS_API int saps_debug_staging_wait(saps_ctx* ctx, int give_up);
+
 /* ---- errors ----------------------------------------------------------------------------------- */
 
 /* Waits for `stream`, then returns in *out_device_status the first error a kernel of this

@@ -70,6 +70,7 @@ _SIGNATURES = {
     "saps_consensus_distance": (_i32, [_vp, _vp, _vp, _vp]),
     "saps_comm_stats": (_i32, [_vp, _vp, _vp, _u64, _f64, _vp]),
     "saps_debug_inject": (_i32, [_vp, _u32, _u32]),
+    "saps_debug_staging_wait": (_i32, [_vp, _i32]),
     "saps_round_host": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp, _vp]),
     "saps_round_pack_host": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "saps_set_host_pipeline": (_i32, [_vp, _u64, _i32]),
@@ -292,6 +293,10 @@ def saps_comm_stats(ctx, bandwidth, pairs, count: int, bits_per_s_per_unit: floa
 
 def saps_debug_inject(ctx, skip_tile: int, spin_limit: int) -> None:
     _check(_lib.saps_debug_inject(ctx, skip_tile, spin_limit), "saps_debug_inject")
+
+
+def saps_debug_staging_wait(ctx, give_up: bool) -> None:
+    _check(_lib.saps_debug_staging_wait(ctx, 1 if give_up else 0), "saps_debug_staging_wait")
 
 
 def saps_round_host(ctx, x_host, g_host, lr, pairs, t, keep_frac, d_x, d_g) -> None:

@@ -242,7 +242,9 @@ __global__ void __launch_bounds__(kThreads) mask_kernel(uint32_t N, uint32_t col
 }
 
 // Receiving side of the exchange (Algorithm 2, merge): one thread per (worker, received entry).
-__global__ void __launch_bounds__(kThreads) unpack_avg_kernel(const UnpackArgs a)
+// The argument block stays in the constant bank (__grid_constant__): src[] is indexed by the block
+// row, and without the qualifier every thread would first copy the whole block to local memory.
+__global__ void __launch_bounds__(kThreads) unpack_avg_kernel(const __grid_constant__ UnpackArgs a)
 {
     const uint32_t src = a.src[blockIdx.y];
     if (src == kNoPeer) return;

@@ -201,8 +201,9 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
     // reads its vectors straight from global memory: same values, and the status word says so)
     bool staged = false;
     if constexpr (BULK) {
-        staged = bulk_bytes != 0 && bulk_wait(shared_address(&s_bar));
-        if (bulk_bytes != 0 && !staged && a.status != nullptr) atomicCAS(a.status, 0, -5 /* SAPS_ERR_TIMEOUT */);
+        staged = bulk_bytes != 0 && !a.staging_give_up && bulk_wait(shared_address(&s_bar));
+        if (bulk_bytes != 0 && !staged && a.status != nullptr && *reinterpret_cast<volatile int*>(a.status) == 0)
+            atomicCAS(a.status, 0, -5 /* SAPS_ERR_TIMEOUT */);
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             if (inb[u]) {

@@ -20,6 +20,7 @@ struct saps_ctx {
     cudaEvent_t ev_before, ev_after;  // optional: recorded around the round kernel
     int gossip_first;       // update order: 0 Algorithm 2, 1 Eq. 7
     int staging;            // SAPS_STAGING_*
+    int staging_give_up;    // test hook of the staged form's bounded wait
     uint32_t spin_limit;    // poll budget of the look-back
     uint32_t skip_tile;     // test hook, 0xFFFFFFFF = off
     double* partials;       // device, for the consensus distance: one double per block of columns
@@ -159,6 +160,7 @@ RoundArgs round_args(const saps_ctx* ctx, float* x, const float* g, float lr, co
     a.tile_count = ctx->ntiles;
     a.gossip_first = ctx->gossip_first;
     a.staging = ctx->staging;
+    a.staging_give_up = ctx->staging_give_up;
     a.out_vals = nullptr;
     a.cap = 0;
     a.tile_cnt = nullptr;
@@ -167,7 +169,7 @@ RoundArgs round_args(const saps_ctx* ctx, float* x, const float* g, float lr, co
     a.ngroups = ctx->ngroups;
     a.out_idx = nullptr;
     a.out_count = nullptr;
-    a.status = nullptr;
+    a.status = static_cast<int*>(ctx->scratch);   // NULL until a call of this context created the scratch
     a.next_cnt = nullptr;
     a.next_group_cnt = nullptr;
     a.clear_group_cnt = nullptr;
@@ -213,6 +215,7 @@ int saps_create_ld(int n, uint64_t N, uint64_t ld, uint64_t seed, saps_ctx** out
     ctx->cap_override = 0;
     ctx->gossip_first = 0;
     ctx->staging = SAPS_STAGING_AUTO;
+    ctx->staging_give_up = 0;
     ctx->spin_limit = kSpinLimit;
     ctx->skip_tile = 0xFFFFFFFFu;
     ctx->partials = nullptr;
@@ -429,6 +432,13 @@ int saps_debug_inject(saps_ctx* ctx, uint32_t skip_tile, uint32_t spin_limit)
     if (ctx == nullptr) return SAPS_ERR_INVALID;
     ctx->skip_tile = skip_tile;
     ctx->spin_limit = spin_limit == 0 ? kSpinLimit : spin_limit;
+    return SAPS_OK;
+}
+
+int saps_debug_staging_wait(saps_ctx* ctx, int give_up)
+{
+    if (ctx == nullptr) return SAPS_ERR_INVALID;
+    ctx->staging_give_up = give_up != 0;
     return SAPS_OK;
 }
 

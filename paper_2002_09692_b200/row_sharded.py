@@ -3,9 +3,11 @@ spread over several GPUs (one process per GPU, `per_rank` consecutive workers ea
 
 A matched pair whose two workers live on the same GPU is averaged in place by the fused
 round.  A pair that straddles two GPUs really exchanges its packed buffer (Algorithm 2:
-ExchangeModelWithPeer): SGD step -> saps_pack -> one send and one receive of `cap` floats
-per such worker (torch.distributed point-to-point, NCCL over NVLink on GPUs) ->
-saps_unpack_avg_rows.  Received buffers land in this GPU's own memory before any kernel
+ExchangeModelWithPeer): the same fused pass that applies the SGD step also writes every
+worker's packed buffer (saps_round_pack; a worker whose peer is remote is a single row of that
+pass, so what it emits is its post-SGD model at the kept coordinates) -> one send and one
+receive of `cap` floats per such worker (torch.distributed point-to-point, NCCL over NVLink on
+GPUs) -> saps_unpack_avg_rows.  Received buffers land in this GPU's own memory before any kernel
 reads them.  Buffers travel at their full capacity `cap` (a few percent more than `count`),
 so no device-to-host read of the count is needed before sending.
 
@@ -78,9 +80,11 @@ class RowShardedGossip:
         buffers of the workers whose peer is remote.  Returns the exchange plan."""
         sb = self.sb
         plan = plan_row_exchange(pairs, self.rank, self.world, self.per_rank)
-        sb.saps_round(self.ctx, x, g, lr, plan.local_pairs, t, keep_frac)
         if plan.transfers:
-            sb.saps_pack(self.ctx, x, t, keep_frac, vals, idx, count)
+            # one pass: SGD step, local averages, and the wire buffers (values before any average)
+            sb.saps_round_pack(self.ctx, x, g, lr, plan.local_pairs, t, keep_frac, vals, idx, count)
+        else:
+            sb.saps_round(self.ctx, x, g, lr, plan.local_pairs, t, keep_frac)
         return plan
 
     def merge(self, x, plan, recv, idx, count, keep_frac):

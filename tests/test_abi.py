@@ -99,6 +99,9 @@ def test_round_rejects_bad_arguments_before_any_launch():
     assert sb._lib.saps_unpack_avg(ctx, fake, None, fake, fake, 0.5, None, None) == sb.SAPS_ERR_INVALID
     assert sb._lib.saps_unpack_avg(ctx, fake, fake, fake, fake, 0.5, sb._pairs([1, 2, 0, 3]), None) == sb.SAPS_ERR_PAIRS
     assert sb._lib.saps_consensus_distance(ctx, fake, None, None) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_debug_staging_wait(None, 1) == sb.SAPS_ERR_INVALID
+    assert sb._lib.saps_debug_staging_wait(ctx, 1) == sb.SAPS_OK
+    assert sb._lib.saps_debug_staging_wait(ctx, 0) == sb.SAPS_OK
     assert sb._lib.saps_set_staging(ctx, 3) == sb.SAPS_ERR_INVALID
     assert sb._lib.saps_set_staging(ctx, -1) == sb.SAPS_ERR_INVALID
     assert sb._lib.saps_set_staging(ctx, sb.SAPS_STAGING_BULK) == sb.SAPS_OK

@@ -205,6 +205,48 @@ def test_bounded_wait_reports_a_timeout_instead_of_hanging(sb):
     sb.saps_destroy(ctx)
 
 
+@pytest.mark.parametrize("N,ld", [(40_000, 40_000), (6_151, 6_152), (2_048, 2_048)])
+def test_staged_round_whose_wait_runs_out_falls_back_to_plain_accesses(sb, N, ld):
+    # The staged form of the fused round waits, bounded, for its bulk copies.  The hook makes that
+    # wait count as run out in every block: the threads then read and write global memory
+    # themselves.  The round, the wire buffer and the next round must still equal the oracle's,
+    # the status word must say SAPS_ERR_TIMEOUT, and the context must work normally afterwards.
+    torch = torch_cuda()
+    n, p, lr, seed = 6, 0.05, 0.1, 41
+    x = synth.gaussian_matrix(n, N, 1.0, seed, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, seed, 1)
+    dx, dg = DeviceMatrix(x, ld), DeviceMatrix(g, ld)
+    ctx = sb.saps_create_ld(n, N, ld, seed)
+    sb.saps_set_staging(ctx, sb.SAPS_STAGING_BULK)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    count = torch.zeros(1, dtype=torch.int32, device="cuda")
+    want = x.copy()
+    pairs = [1, 0, 3, 2, 4, 5]                      # two pairs and two single workers
+    for t, give_up, emit in ((1, True, True), (2, True, False), (3, False, True), (4, False, False)):
+        sb.saps_debug_staging_wait(ctx, give_up)
+        a = want.copy()
+        oracle.sgd(a, g, lr)
+        if emit:
+            sb.saps_round_pack(ctx, dx.ptr, dg.ptr, lr, pairs, t, p, vals, idx, count)
+        else:
+            sb.saps_round(ctx, dx.ptr, dg.ptr, lr, pairs, t, p)
+        torch.cuda.synchronize()
+        assert sb.saps_status(ctx) == (sb.SAPS_ERR_TIMEOUT if give_up else 0), (t, give_up)
+        m = oracle.gossip_round(want, g, lr, pairs, seed, t, p)
+        assert_bits_equal(dx.host(), want, f"round {t}, wait given up: {give_up}")
+        if emit:
+            kept = np.nonzero(m)[0]
+            c = int(count.cpu().numpy().view(np.uint32)[0])
+            assert c == len(kept)
+            assert (idx[:c].cpu().numpy().view(np.uint32) == kept.astype(np.uint32)).all()
+            assert_bits_equal(vals[:, :c].cpu().numpy(), a[:, kept], f"wire buffer of round {t}")
+    assert dx.canaries_intact() and dg.canaries_intact()
+    assert_bits_equal(dg.host(), g, "gradient must not change")
+    sb.saps_destroy(ctx)
+
+
 def test_row_sharded_round_emulated_on_one_gpu(sb):
     # Two "ranks" of 4 workers each, run one after the other on this GPU; the transfer between
     # them is a device copy of the packed rows.  The result must equal the single-context round.
