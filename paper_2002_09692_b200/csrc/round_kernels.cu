@@ -99,6 +99,15 @@ __device__ __forceinline__ bool bulk_wait(uint32_t bar)
     return done != 0;
 }
 
+// Programmatic dependent launch: consecutive rounds in a stream are launched so that the next
+// round's blocks may be set up, and hash their columns, while the last blocks of this round still
+// run.  grid_dependents_may_start() lets the next launch begin once every block of this grid has
+// started; wait_for_previous_grid() returns when the grid before this one in the stream (and with
+// it every earlier one) has completed and its writes are visible.  A block touches global memory
+// only behind that wait.  After any other kind of predecessor the wait returns at once.
+__device__ __forceinline__ void grid_dependents_may_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void wait_for_previous_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // GOSSIP_FIRST selects the order of Eq. 7 (average the current models, then subtract the
 // gradient step) instead of Algorithm 2's (SGD step first, then average).
 // BULK (VEC = 4 with gradients only): the row pieces travel through shared memory by bulk copies.
@@ -109,6 +118,7 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
     constexpr int U = kTileCols / (kThreads * VEC);
     constexpr int kWarps = kThreads / 32;
     const int tid = threadIdx.x;
+    grid_dependents_may_start();
     const uint32_t tile = a.tile_begin + blockIdx.x;
     const uint32_t ra = a.groups.a[blockIdx.y];
     const uint32_t rb_raw = a.groups.b[blockIdx.y];
@@ -138,6 +148,7 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
         }
         __syncthreads();
         if (tid == 0 && bulk_bytes != 0) {
+            wait_for_previous_grid();
             const uint32_t pieces = paired ? 4u : 2u;
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(pieces * bulk_bytes) : "memory");
             bulk_load(s_stage[0], xa + col_tile, bulk_bytes, bar);
@@ -153,6 +164,7 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
     bool inb[U];
     uint32_t col[U];
 
+    if constexpr (!BULK) wait_for_previous_grid();
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const uint64_t k = col_tile + (uint64_t)(u * kThreads + tid) * VEC;
@@ -171,13 +183,15 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
     // The rank offset of the tile = kept columns in all earlier tiles: whole groups of tiles from
     // the group sums, the rest tile by tile; every thread takes a share (one load, seldom more),
     // the block adds them up further down.  Placed behind the model loads, so that waiting for
-    // these few values never delays them.
+    // these few values never delays them.  (The counts may have been written by the previous
+    // round's kernel while this one was already being set up: plain L2 loads, not the read-only path.)
     uint32_t excl_part = 0;
-    if constexpr (EMIT) {
+    auto load_rank_offset_share = [&]() {
         const uint32_t g = tile >> a.group_shift;
-        for (uint32_t j = tid; j < g; j += kThreads) excl_part += __ldg(a.group_cnt + j);
-        for (uint32_t j = (g << a.group_shift) + tid; j < tile; j += kThreads) excl_part += __ldg(a.tile_cnt + j);
-    }
+        for (uint32_t j = tid; j < g; j += kThreads) excl_part += __ldcg(a.group_cnt + j);
+        for (uint32_t j = (g << a.group_shift) + tid; j < tile; j += kThreads) excl_part += __ldcg(a.tile_cnt + j);
+    };
+    if constexpr (EMIT && !BULK) load_rank_offset_share();
 
     uint32_t bits[U];
 #pragma unroll
@@ -201,6 +215,9 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
     // reads its vectors straight from global memory: same values, and the status word says so)
     bool staged = false;
     if constexpr (BULK) {
+        // the columns are hashed by now; everything from here on reads or writes global memory
+        wait_for_previous_grid();
+        if constexpr (EMIT) load_rank_offset_share();
         staged = bulk_bytes != 0 && !a.staging_give_up && bulk_wait(shared_address(&s_bar));
         if (bulk_bytes != 0 && !staged && a.status != nullptr && *reinterpret_cast<volatile int*>(a.status) == 0)
             atomicCAS(a.status, 0, -5 /* SAPS_ERR_TIMEOUT */);
@@ -460,7 +477,7 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
         if (tile == 0 && blockIdx.y == 0) {
             __shared__ uint32_t s_tot[kWarps];
             uint32_t t = 0;
-            for (uint32_t j = tid; j < a.ngroups; j += kThreads) t += __ldg(a.group_cnt + j);
+            for (uint32_t j = tid; j < a.ngroups; j += kThreads) t += __ldcg(a.group_cnt + j);
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, d);
             if ((tid & 31) == 0) s_tot[tid >> 5] = t;
@@ -482,6 +499,25 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
 // barriers of the staged form cost more than its better use of the memory system gains.
 constexpr uint64_t kBulkMinBlocks = 4096;
 
+// Launched as a programmatic dependent of whatever kernel precedes it in the stream: after another
+// round kernel its blocks may start early (they wait for that grid before they touch memory),
+// after anything else the launch is an ordinary one.
+template <typename Kernel>
+cudaError_t launch_dependent(Kernel kernel, dim3 grid, const RoundArgs& a, cudaStream_t stream)
+{
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
 template <int VEC, bool HAS_G, bool EMIT, bool GOSSIP_FIRST>
 cudaError_t launch_variant(const RoundArgs& a, cudaStream_t stream)
 {
@@ -492,16 +528,14 @@ cudaError_t launch_variant(const RoundArgs& a, cudaStream_t stream)
         const bool bulk = a.staging == 2 || (a.staging == 0 && (uint64_t)a.tile_count * a.groups.count >= kBulkMinBlocks);
         if (bulk) {
             auto kernel = round_kernel<VEC, HAS_G, EMIT, GOSSIP_FIRST, true>;
-            // once per process and kernel: let five blocks of 32 KB share an SM
+            // once per process and kernel: let several blocks of 33 KB share an SM
             static const cudaError_t carve =
                 cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
             if (carve != cudaSuccess) return carve;
-            kernel<<<grid, kThreads, 0, stream>>>(a);
-            return cudaGetLastError();
+            return launch_dependent(kernel, grid, a, stream);
         }
     }
-    round_kernel<VEC, HAS_G, EMIT, GOSSIP_FIRST, false><<<grid, kThreads, 0, stream>>>(a);
-    return cudaGetLastError();
+    return launch_dependent(round_kernel<VEC, HAS_G, EMIT, GOSSIP_FIRST, false>, grid, a, stream);
 }
 
 template <int VEC>
