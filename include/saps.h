@@ -326,9 +326,10 @@ SAPS_API int saps_round_pack_host(saps_ctx* ctx, float* x_host, const float* g_h
                                   uint32_t* d_count);
 
 /* Tuning of the copy/compute pipeline behind the two host-buffer entry points: columns per
- * chunk (rounded up to whole 2048-column tiles; default 1,048,576) and the number of streams
- * that copy chunks in and run the round on them (1..6, default 3; results always leave on one
- * further stream).  0 leaves a setting as it is.  Results do not depend on either. */
+ * chunk (rounded up to whole 2048-column tiles; default 1,048,576; the last chunks of a row halve
+ * down to 65,536 columns, so that little is left to do once the last copy-in has landed) and the
+ * number of streams that copy chunks in and run the round on them (1..6, default 3; results
+ * always leave on one further stream).  0 leaves a setting as it is.  Results do not depend on either. */
 SAPS_API int saps_set_host_pipeline(saps_ctx* ctx, uint64_t chunk_columns, int lanes);
 
 /* ---- consensus and communication metrics -------------------------------------------------------- */

@@ -806,10 +806,18 @@ int round_host_impl(saps_ctx* ctx, float* x_host, const float* g_host, float lr,
         for (int l = 1; l < lanes; ++l)
             failed |= cudaStreamWaitEvent(ctx->lane_stream[l], ctx->scan_event, 0) != cudaSuccess;
     }
+    // Chunks of host_chunk_tiles column tiles; towards the end they halve (down to kMinChunkTiles),
+    // because what follows the last copy-in (its kernel and its copy-out) is not overlapped with
+    // anything and should be short.
+    constexpr uint32_t kMinChunkTiles = 32;
     const uint32_t tiles_per_chunk = ctx->host_chunk_tiles;
     int lane = 0;
-    for (uint32_t tb = 0; tb < ctx->ntiles && !failed; tb += tiles_per_chunk, lane = (lane + 1) % lanes) {
-        const uint32_t tc = ctx->ntiles - tb < tiles_per_chunk ? ctx->ntiles - tb : tiles_per_chunk;
+    uint32_t tc = 0;
+    for (uint32_t tb = 0; tb < ctx->ntiles && !failed; tb += tc, lane = (lane + 1) % lanes) {
+        const uint32_t remaining = ctx->ntiles - tb;
+        const uint32_t half = (remaining + 1) / 2;
+        const uint32_t tail = half >= kMinChunkTiles ? half : remaining;   // fewer than two small chunks left: one
+        tc = tail < tiles_per_chunk ? tail : tiles_per_chunk;
         const uint64_t c0 = (uint64_t)tb * kTileCols;
         const uint64_t c1 = c0 + (uint64_t)tc * kTileCols < N ? c0 + (uint64_t)tc * kTileCols : N;
         const size_t width = (size_t)(c1 - c0) * sizeof(float);

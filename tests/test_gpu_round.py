@@ -350,6 +350,49 @@ def test_run_rounds_pack_emits_every_round(sb):
     sb.saps_destroy(ctx)
 
 
+@pytest.mark.parametrize("n,N,ld,emit", [(4, 5_000, 5_000, True), (6, 2_050, 2_052, True), (4, 700, 700, False),
+                                         (8, 9_001, 9_001, True)])
+def test_many_small_rounds_back_to_back(sb, n, N, ld, emit):
+    # Launches of a handful of blocks, 150 of them in one scheduler call: consecutive round
+    # kernels are launched as programmatic dependents, so with grids this small several of them
+    # are resident at once, each waiting for its predecessor before it touches memory, and the
+    # per-tile mask counts pass from each kernel to the next.  Every round's count and the final
+    # model and wire buffer must equal the oracle's.
+    torch = torch_cuda()
+    T, p, lr, seed = 150, 0.08, 0.05, 77
+    x = synth.gaussian_matrix(n, N, 1.0, seed, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, seed, 1)
+    rng = synth.matching_rng(seed)
+    pairs_list = np.asarray([synth.random_perfect_matching(n, rng) for _ in range(T)], dtype=np.int32)
+    dx, dg = DeviceMatrix(x, ld), DeviceMatrix(g, ld)
+    ctx = sb.saps_create_ld(n, N, ld, seed)
+    cap = sb.saps_pack_capacity(ctx, p)
+    vals = torch.zeros(n, cap, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(cap, dtype=torch.int32, device="cuda")
+    counts = torch.zeros(T, dtype=torch.int32, device="cuda")
+    if emit:
+        sb.saps_run_rounds_pack(ctx, dx.ptr, dg.ptr, lr, 1, T, p, vals, idx, counts, pairs_list=pairs_list)
+    else:
+        sb.saps_run_rounds(ctx, dx.ptr, dg.ptr, lr, 1, T, p, pairs_list=pairs_list)
+    torch.cuda.synchronize()
+    assert sb.saps_status(ctx) == 0
+    want = x.copy()
+    got_counts = counts.cpu().numpy().view(np.uint32)
+    for t in range(1, T + 1):
+        a = want.copy()
+        oracle.sgd(a, g, lr)
+        m = oracle.gossip_round(want, g, lr, pairs_list[t - 1], seed, t, p)
+        if emit:
+            assert int(got_counts[t - 1]) == int(m.sum()), t
+    assert_bits_equal(dx.host(), want, "150 small rounds in one call")
+    if emit:
+        kept = np.nonzero(m)[0]
+        assert (idx[:len(kept)].cpu().numpy().view(np.uint32) == kept.astype(np.uint32)).all()
+        assert_bits_equal(vals[:, :len(kept)].cpu().numpy(), a[:, kept], "wire buffer of the last round")
+    assert dx.canaries_intact() and dg.canaries_intact()
+    sb.saps_destroy(ctx)
+
+
 def test_scheduler_loop_captured_in_a_cuda_graph_and_replayed(sb):
     # Every device operation of the library is enqueued on the caller's stream and, after the
     # first use of a context, nothing is allocated: a round loop can be captured in a CUDA graph.
