@@ -79,6 +79,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--no-small-loop", action="store_true")
+    ap.add_argument("--dist-backend", default="nccl", choices=["nccl", "gloo"],
+                    help="process-group backend for N > 1 (barrier and max over ranks only; the round needs no "
+                         "collective).  gloo lets the multi-rank branch run where several ranks share one GPU")
     return ap.parse_args()
 
 
@@ -162,15 +165,17 @@ def oracle_step(oracle, ps, x, g, w, B, R, t, keep_frac, b_thres, t_thres, cap):
     oracle.pair_average(x, np.asarray(pairs, dtype=np.int32), m)
 
 
-def oracle_sample(w):
-    """Columns the oracle runs on per step: the whole model when it has at most
-    ORACLE_MAX_COLUMNS columns (the benchmark's default workload has), else the first
-    ORACLE_MAX_COLUMNS, with rounds/s scaled in proportion."""
+def oracle_sample(w, world=1):
+    """Columns the oracle runs on per step and the fraction of the whole job they are.  At N ranks
+    the job is N column shards of w.N columns each (weak scaling); the oracle runs one shard, or
+    its first ORACLE_MAX_COLUMNS columns when the shard is larger, and rounds/s is scaled in
+    proportion.  On one GPU with the benchmark's default workload nothing is scaled."""
     cols = min(w.N, ORACLE_MAX_COLUMNS)
-    if cols == w.N:
-        return cols, f"all {w.N} columns of all {w.n} workers per step (nothing scaled)"
-    return cols, (f"first {cols} of {w.N} columns of all {w.n} workers per step; "
-                  f"rounds/s scaled by {cols}/{w.N}")
+    total = w.N * world
+    if cols == total:
+        return cols, 1.0, f"all {w.N} columns of all {w.n} workers per step (nothing scaled)"
+    return cols, cols / total, (f"first {cols} of {total} columns ({world} shard(s) of {w.N}) of all {w.n} workers "
+                                f"per step; rounds/s scaled by {cols}/{total}")
 
 
 def run_reference(args):
@@ -183,7 +188,7 @@ def run_reference(args):
     from oracle import peer_selection as ps
     from paper_2002_09692_b200 import synth
     w = synth.WORKLOADS[args.workload]
-    cols, sample = oracle_sample(w)
+    cols, frac, sample = oracle_sample(w, max(1, args.gpus))
     x = synth.gaussian_matrix(w.n, cols, w.x_std, w.seed, 0)
     g = synth.gaussian_matrix(w.n, cols, w.g_std, w.seed, 1)
     B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
@@ -200,12 +205,12 @@ def run_reference(args):
         t += 1
     dt = time.perf_counter() - t0
     ms = dt / args.steps * 1e3
-    value = (cols / w.N) / (dt / args.steps)
+    value = frac / (dt / args.steps)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": workload_config(w, args.keep_frac, 1),
+        "config": workload_config(w, args.keep_frac, max(1, args.gpus)),
         "sample_columns": cols,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -244,10 +249,14 @@ def run_ours(args):
     rank, world, local = dist_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    local = local % torch.cuda.device_count()
     torch.cuda.set_device(local)
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if args.dist_backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group("gloo")
 
     w = synth.WORKLOADS[args.workload]
     n, N, p = w.n, w.N, args.keep_frac
@@ -384,8 +393,11 @@ def run_ours(args):
     # what was timed is also what is right: the next step of the same sequence (same context, so
     # its per-tile counts come from the previous kernel's run-ahead exactly as in the timed
     # steps), replayed by the CPU oracle on a few sampled rows (outside every timed region)
-    if rank == 0 and not args.no_verify:
-        result["verified"] = verify_step(sb, ctx, w, B, t, p, x, g, vals, idx, count, stream)
+    if not args.no_verify:
+        if rank == 0:
+            result["verified"] = verify_step(sb, ctx, w, B, t, p, x, g, vals, idx, count, stream)
+        else:               # the other ranks take the same step, so that every rank's matching sequence stays the same
+            step(t)
     t += 1
 
     # the other entry points of the path, each timed alone on the same resident inputs (context
@@ -640,7 +652,7 @@ def measure_cpu_baseline(args, w, x_dev, g_dev):
     import oracle
     from oracle import peer_selection as ps
     from paper_2002_09692_b200 import synth
-    cols, sample = oracle_sample(w)
+    cols, frac, sample = oracle_sample(w)
     x = np.ascontiguousarray(x_dev[:, :cols].cpu().numpy())
     g = np.ascontiguousarray(g_dev[:, :cols].cpu().numpy())
     B = synth.bandwidth_matrix(w.n, *w.bw_range, seed=w.seed)
@@ -652,7 +664,7 @@ def measure_cpu_baseline(args, w, x_dev, g_dev):
     for r in range(rounds):
         oracle_step(oracle, ps, x, g, w, B, R, 2 + r, args.keep_frac, b_thres, t_thres, cols)
     dt = (time.perf_counter() - t0) / rounds
-    return {"value": (cols / w.N) / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+    return {"value": frac / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
             "host_cores_present": os.cpu_count(), "ms_per_round": dt * 1e3,
             "sample": f"{rounds} rounds (after 1 warm-up) over " + sample}
 

@@ -43,10 +43,15 @@ def test_reference_arm_runs_the_whole_default_workload():
     sys.path.insert(0, ROOT)
     import bench
     from paper_2002_09692_b200 import synth
-    cols, sample = bench.oracle_sample(synth.WORKLOADS["vgg16"])
-    assert cols == synth.WORKLOADS["vgg16"].N and "nothing scaled" in sample
-    cols, sample = bench.oracle_sample(synth.WORKLOADS["gpt2s"])
+    cols, frac, sample = bench.oracle_sample(synth.WORKLOADS["vgg16"])
+    assert cols == synth.WORKLOADS["vgg16"].N and frac == 1.0 and "nothing scaled" in sample
+    cols, frac, sample = bench.oracle_sample(synth.WORKLOADS["gpt2s"])
     assert cols == bench.ORACLE_MAX_COLUMNS < synth.WORKLOADS["gpt2s"].N and "scaled by" in sample
+    assert frac == cols / synth.WORKLOADS["gpt2s"].N
+    # at N ranks the job is N column shards; the oracle runs one and says what fraction that is
+    cols, frac, sample = bench.oracle_sample(synth.WORKLOADS["vgg16"], 4)
+    assert cols == synth.WORKLOADS["vgg16"].N and frac == 0.25 and "4 shard(s)" in sample
+    assert bench.workload_config(synth.WORKLOADS["vgg16"], 0.01, 4)["sharding"].startswith("column shards")
     small = bench.workload_config(synth.WORKLOADS["resnet20"], 0.01, 1)
     assert "L2-resident" in small["l2"]
     big = bench.workload_config(synth.WORKLOADS["vgg16"], 0.01, 1)
