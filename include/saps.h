@@ -126,6 +126,22 @@ SAPS_API int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, 
                     uint64_t t, double keep_frac, float* out_vals, uint32_t* out_idx,
                     uint32_t* out_count, void* stream);
 
+/* saps_round_pack with one destination per worker instead of one [n, cap] matrix (Algorithm 2,
+ * ExchangeModelWithPeer, for workers spread over several GPUs): out_rows is a DEVICE array of n
+ * pointers; worker i's packed values go to out_rows[i][0 .. count) (room for cap floats), and a
+ * NULL entry means worker i's values are not wanted.  A destination may be any address this GPU
+ * can store to: with peer access enabled, the receive buffer of the worker's peer on another GPU;
+ * the kernel then writes the wire buffer straight into the receiver's memory with ordinary
+ * stores while the same pass streams the model, and no separate transfer follows.  The receiver
+ * may read it once this call's stream work has completed and that fact has reached it (a stream
+ * synchronisation on this side followed by a host-side barrier, or an interprocess event).
+ * out_idx, out_count as in saps_round_pack (local device memory).  The table is read by the
+ * kernel: keep it unchanged until the call's stream work has completed. */
+SAPS_API int saps_round_pack_rows(saps_ctx* ctx, float* x, const float* g, float lr,
+                                  const int32_t* pairs, uint64_t t, double keep_frac,
+                                  float* const* out_rows, uint32_t* out_idx, uint32_t* out_count,
+                                  void* stream);
+
 /* The emitting entry points need the number of kept columns per column tile before the fused
  * kernel runs (a block derives the ranks of its kept columns from the counts of all earlier
  * tiles).  By default that kernel also counts them for round t+1 while it streams round t (the

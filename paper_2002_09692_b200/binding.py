@@ -51,6 +51,7 @@ _SIGNATURES = {
     "saps_mask": (_i32, [_vp, _u64, _f64, _vp, _vp]),
     "saps_round": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp]),
     "saps_round_pack": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp, _vp, _vp, _vp]),
+    "saps_round_pack_rows": (_i32, [_vp, _vp, _vp, _f32, _vp, _u64, _f64, _vp, _vp, _vp, _vp]),
     "saps_pack_capacity": (_u64, [_vp, _f64]),
     "saps_set_pack_capacity": (_i32, [_vp, _u64]),
     "saps_pack": (_i32, [_vp, _vp, _u64, _f64, _vp, _vp, _vp, _vp]),
@@ -170,6 +171,12 @@ def saps_round(ctx, x, g, lr, pairs, t, keep_frac, stream=None) -> None:
 def saps_round_pack(ctx, x, g, lr, pairs, t, keep_frac, out_vals, out_idx, out_count, stream=None) -> None:
     _check(_lib.saps_round_pack(ctx, _ptr(x), _ptr(g), lr, _pairs(pairs), t, keep_frac, _ptr(out_vals),
                                 _ptr(out_idx), _ptr(out_count), _stream(stream)), "saps_round_pack")
+
+
+def saps_round_pack_rows(ctx, x, g, lr, pairs, t, keep_frac, out_rows, out_idx, out_count, stream=None) -> None:
+    """out_rows: device array of n 64-bit addresses (e.g. an int64 tensor), one destination per worker."""
+    _check(_lib.saps_round_pack_rows(ctx, _ptr(x), _ptr(g), lr, _pairs(pairs), t, keep_frac, _ptr(out_rows),
+                                     _ptr(out_idx), _ptr(out_count), _stream(stream)), "saps_round_pack_rows")
 
 
 def saps_pack_capacity(ctx, keep_frac: float) -> int:

@@ -78,7 +78,8 @@ struct RoundArgs {
     // columns start at the number of kept columns in all earlier tiles.  That number is summed by
     // the block itself from two small arrays: the kept columns per tile, and their sums over
     // groups of 2^group_shift consecutive tiles.
-    float* out_vals;
+    float* out_vals;             // [n, cap], or NULL when out_rows is given
+    float* const* out_rows;      // device array of n destinations (NULL entries: not emitted), or NULL
     uint32_t cap;
     const uint32_t* tile_cnt;    // kept columns per tile, this round
     const uint32_t* group_cnt;   // the same summed over every group of tiles

@@ -258,7 +258,19 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
     uint32_t rank[U];       // EMIT only: rank of this thread's first kept column
     uint32_t total = 0;     // EMIT only: kept columns in the vector part of the tile
     uint32_t excl = 0;      // EMIT only: kept columns in all earlier tiles
+    // EMIT only: where the two workers' packed values go.  Rows of one [n, cap] matrix, or, with
+    // a table of destinations, any address this GPU can store to (a peer GPU's receive buffer,
+    // for one: the stores then cross the link while the pass streams on); NULL = not wanted.
+    float* dst_a = nullptr;
+    float* dst_b = nullptr;
     if constexpr (EMIT) {
+        if (a.out_rows != nullptr) {
+            dst_a = a.out_rows[ra];
+            dst_b = a.out_rows[rb];
+        } else {
+            dst_a = a.out_vals + (size_t)ra * a.cap;
+            dst_b = a.out_vals + (size_t)rb * a.cap;
+        }
         // Two counts travel in one word (16 bits each: a tile keeps at most 2048 columns), so one
         // warp scan and one pass over the warps' totals serve two of the thread's vectors.
         static_assert(U % 2 == 0, "vectors are ranked two at a time");
@@ -348,8 +360,8 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
                 for (int c = 0; c < VEC; ++c) {
                     if ((bits[u] >> c) & 1u) {
                         if (r < a.cap) {
-                            a.out_vals[(size_t)ra * a.cap + r] = va[u].v[c];
-                            if (paired) a.out_vals[(size_t)rb * a.cap + r] = vb[u].v[c];
+                            if (dst_a != nullptr) dst_a[r] = va[u].v[c];
+                            if (paired && dst_b != nullptr) dst_b[r] = vb[u].v[c];
                         }
                         ++r;
                     }
@@ -450,8 +462,8 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
                     for (uint32_t q = nfull; q < k; ++q) r += column_kept(a.col_offset + q, a.key) ? 1u : 0u;
                     if (r < a.cap) {
                         if (blockIdx.y == 0 && a.out_idx != nullptr) a.out_idx[r] = a.col_offset + k;
-                        a.out_vals[(size_t)ra * a.cap + r] = pa;
-                        if (paired) a.out_vals[(size_t)rb * a.cap + r] = pb;
+                        if (dst_a != nullptr) dst_a[r] = pa;
+                        if (paired && dst_b != nullptr) dst_b[r] = pb;
                     }
                 }
             }

@@ -162,6 +162,7 @@ RoundArgs round_args(const saps_ctx* ctx, float* x, const float* g, float lr, co
     a.staging = ctx->staging;
     a.staging_give_up = ctx->staging_give_up;
     a.out_vals = nullptr;
+    a.out_rows = nullptr;
     a.cap = 0;
     a.tile_cnt = nullptr;
     a.group_cnt = nullptr;
@@ -598,6 +599,27 @@ int saps_round_pack(saps_ctx* ctx, float* x, const float* g, float lr, const int
     rc = prepare_emission(ctx, t, keep_frac, cap, out_idx, out_count, out_vals, (cudaStream_t)stream, &a);
     if (rc != SAPS_OK) return rc;
     // the fused round writes the kept columns and each worker's kept values at their ranks
+    rc = timed_round(ctx, a, true, (cudaStream_t)stream);
+    if (rc != SAPS_OK) ctx->ahead_valid = false;
+    return rc;
+}
+
+int saps_round_pack_rows(saps_ctx* ctx, float* x, const float* g, float lr, const int32_t* pairs, uint64_t t,
+                         double keep_frac, float* const* out_rows, uint32_t* out_idx, uint32_t* out_count,
+                         void* stream)
+{
+    int rc = check_round_args(ctx, x, g, lr, t, keep_frac);
+    if (rc != SAPS_OK) return rc;
+    if (out_rows == nullptr || out_count == nullptr) return SAPS_ERR_INVALID;
+    rc = check_pairs(ctx->n, pairs);
+    if (rc != SAPS_OK) return rc;
+    const RoundKey key = make_key(ctx->seed, t, keep_frac);
+    const uint32_t cap = (uint32_t)saps_pack_capacity(ctx, keep_frac);
+    const RowGroups rg = make_groups(ctx->n, pairs, true);
+    RoundArgs a = round_args(ctx, x, g, lr, rg, key);
+    rc = prepare_emission(ctx, t, keep_frac, cap, out_idx, out_count, nullptr, (cudaStream_t)stream, &a);
+    if (rc != SAPS_OK) return rc;
+    a.out_rows = out_rows;
     rc = timed_round(ctx, a, true, (cudaStream_t)stream);
     if (rc != SAPS_OK) ctx->ahead_valid = false;
     return rc;

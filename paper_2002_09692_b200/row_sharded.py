@@ -12,6 +12,14 @@ reads them.  Buffers travel at their full capacity `cap` (a few percent more tha
 so no device-to-host read of the count is needed before sending.
 
 `plan_row_exchange` is pure host logic; `exchange_rows` is the only communication step.
+
+Direct form (`destination_table`, `RowShardedGossip.local_step_direct`): where the GPUs can store
+into one another's memory (peer access over NVLink; the receive buffers mapped into every process,
+e.g. through CUDA IPC handles or a symmetric-memory allocation), the fused pass writes each
+remote-peer worker's packed values straight into the receiving rank's buffer
+(saps_round_pack_rows) and no transfer step follows: only "my pass has finished" has to reach the
+peer (stream synchronisation, then a barrier of the process group) before it merges.  That form
+has run with both ranks' buffers on one GPU only.
 """
 from __future__ import annotations
 
@@ -45,6 +53,19 @@ def plan_row_exchange(pairs, rank: int, world: int, per_rank: int) -> RowExchang
             transfers.append((r, j // per_rank, min(lo + r, j)))
             src_rows.append(r)
     return RowExchangePlan(tuple(local_pairs), tuple(transfers), tuple(src_rows))
+
+
+def destination_table(plan: RowExchangePlan, pairs, rank: int, per_rank: int, recv_base_of_rank, cap: int):
+    """Per local worker, the address its packed values should be written to (for
+    saps_round_pack_rows): row j of rank q's receive buffer when its peer is local row j of rank q
+    (recv_base_of_rank[q] is the address of that [per_rank, cap] fp32 buffer as THIS process sees
+    it), 0 when the peer is local (nothing to send).  The receiver finds the buffer of the worker
+    that local row j is paired with in row j, which is what plan.src_rows says."""
+    table = [0] * per_rank
+    for r, peer_rank, _tag in plan.transfers:
+        j = int(pairs[rank * per_rank + r]) - peer_rank * per_rank
+        table[r] = int(recv_base_of_rank[peer_rank]) + 4 * cap * j
+    return table
 
 
 def exchange_rows(send, recv, plan: RowExchangePlan, group=None) -> None:
@@ -83,6 +104,22 @@ class RowShardedGossip:
         if plan.transfers:
             # one pass: SGD step, local averages, and the wire buffers (values before any average)
             sb.saps_round_pack(self.ctx, x, g, lr, plan.local_pairs, t, keep_frac, vals, idx, count)
+        else:
+            sb.saps_round(self.ctx, x, g, lr, plan.local_pairs, t, keep_frac)
+        return plan
+
+    def local_step_direct(self, x, g, lr, pairs, t, keep_frac, recv_base_of_rank, table_dev, idx, count):
+        """As local_step, but the packed values of the workers whose peer is remote are written by
+        the fused pass itself into the peers' receive buffers.  table_dev: device int64 tensor of
+        per_rank entries that this call fills (it must stay untouched until the pass has run)."""
+        import torch
+        sb = self.sb
+        plan = plan_row_exchange(pairs, self.rank, self.world, self.per_rank)
+        if plan.transfers:
+            cap = sb.saps_pack_capacity(self.ctx, keep_frac)
+            table = destination_table(plan, pairs, self.rank, self.per_rank, recv_base_of_rank, cap)
+            table_dev.copy_(torch.tensor(table, dtype=torch.int64), non_blocking=False)
+            sb.saps_round_pack_rows(self.ctx, x, g, lr, plan.local_pairs, t, keep_frac, table_dev, idx, count)
         else:
             sb.saps_round(self.ctx, x, g, lr, plan.local_pairs, t, keep_frac)
         return plan

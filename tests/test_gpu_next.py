@@ -247,9 +247,12 @@ def test_staged_round_whose_wait_runs_out_falls_back_to_plain_accesses(sb, N, ld
     sb.saps_destroy(ctx)
 
 
-def test_row_sharded_round_emulated_on_one_gpu(sb):
+@pytest.mark.parametrize("direct", [False, True])
+def test_row_sharded_round_emulated_on_one_gpu(sb, direct):
     # Two "ranks" of 4 workers each, run one after the other on this GPU; the transfer between
-    # them is a device copy of the packed rows.  The result must equal the single-context round.
+    # them is a device copy of the packed rows, or (direct) the fused pass of each rank writes
+    # its packed rows straight into the other rank's receive buffer through a table of
+    # destinations.  The result must equal the single-context round.
     torch = torch_cuda()
     from paper_2002_09692_b200.row_sharded import RowShardedGossip
     world, per_rank, N, p, lr, seed = 2, 4, 30_000, 0.05, 0.05, 33
@@ -264,18 +267,28 @@ def test_row_sharded_round_emulated_on_one_gpu(sb):
     cap = sb.saps_pack_capacity(ranks[0].ctx, p)
     bufs = [dict(vals=torch.zeros(per_rank, cap, device="cuda"), recv=torch.zeros(per_rank, cap, device="cuda"),
                  idx=torch.zeros(cap, dtype=torch.int32, device="cuda"),
+                 table=torch.zeros(per_rank, dtype=torch.int64, device="cuda"),
                  count=torch.zeros(1, dtype=torch.int32, device="cuda")) for _ in range(world)]
     want = x.copy()
     crossed = 0
     for t in range(1, 6):
         pairs = synth.random_perfect_matching(n, rng)
-        plans = [ranks[r].local_step(dxs[r].ptr, dgs[r].ptr, lr, pairs, t, p, bufs[r]["vals"], bufs[r]["idx"],
-                                     bufs[r]["count"]) for r in range(world)]
-        for r in range(world):                              # the wire: each packed row goes to its peer's rank
-            for row, peer, _tag in plans[r].transfers:
-                j = int(pairs[r * per_rank + row])
-                bufs[peer]["recv"][j - peer * per_rank].copy_(bufs[r]["vals"][row])
-                crossed += 1
+        if direct:
+            bases = [bufs[r]["recv"].data_ptr() for r in range(world)]
+            for b in bufs:
+                b["recv"].fill_(float("nan"))               # nothing stale may be averaged in
+            plans = [ranks[r].local_step_direct(dxs[r].ptr, dgs[r].ptr, lr, pairs, t, p, bases, bufs[r]["table"],
+                                                bufs[r]["idx"], bufs[r]["count"]) for r in range(world)]
+            torch.cuda.synchronize()                        # "my pass has finished" reaches the peer
+            crossed += sum(len(pl.transfers) for pl in plans)
+        else:
+            plans = [ranks[r].local_step(dxs[r].ptr, dgs[r].ptr, lr, pairs, t, p, bufs[r]["vals"], bufs[r]["idx"],
+                                         bufs[r]["count"]) for r in range(world)]
+            for r in range(world):                          # the wire: each packed row goes to its peer's rank
+                for row, peer, _tag in plans[r].transfers:
+                    j = int(pairs[r * per_rank + row])
+                    bufs[peer]["recv"][j - peer * per_rank].copy_(bufs[r]["vals"][row])
+                    crossed += 1
         for r in range(world):
             ranks[r].merge(dxs[r].ptr, plans[r], bufs[r]["recv"], bufs[r]["idx"], bufs[r]["count"], p)
         oracle.gossip_round(want, g, lr, pairs, seed, t, p)

@@ -182,6 +182,57 @@ def test_round_pack_emits_what_each_worker_sends(sb, N, ld, p, has_g):
     assert dx.canaries_intact()
 
 
+@pytest.mark.parametrize("N,ld", [(7, 7), (2050, 2052), (40_003, 40_032), (40_003, 40_003), (6 * 2048, 6 * 2048)])
+@pytest.mark.parametrize("p", [0.05, 1.0])
+def test_round_pack_rows_writes_each_worker_to_its_own_destination(sb, N, ld, p):
+    # Per-worker destinations (the form that lets a pass store its wire buffers straight into the
+    # receivers' memory): every worker's packed values must land, bit for bit, at the address its
+    # table entry names and nowhere else; a worker with a NULL entry emits nothing; the model,
+    # the index list and the count are those of the ordinary emitting round.
+    torch = torch_cuda()
+    n = 6
+    pairs = [1, 0, 2, 5, 4, 3]                 # workers 2 and 4 have no peer
+    x = synth.gaussian_matrix(n, N, 1.0, 19, 0)
+    g = synth.gaussian_matrix(n, N, 0.01, 19, 1)
+    dx, dg = DeviceMatrix(x, ld), DeviceMatrix(g, ld)
+    ctx = sb.saps_create_ld(n, N, ld, 19)
+    cap = sb.saps_pack_capacity(ctx, p)
+    # one arena, rows handed out in a scrambled order with a guard stretch behind each
+    slot = cap + 16
+    arena = torch.full((n * slot,), 123.0, dtype=torch.float32, device="cuda")
+    order = [3, 0, 5, 1, 4, 2]
+    skipped = 4
+    table = [0 if i == skipped else arena.data_ptr() + 4 * slot * order[i] for i in range(n)]
+    d_table = torch.tensor(table, dtype=torch.int64, device="cuda")
+    idx = torch.full((cap,), -1, dtype=torch.int32, device="cuda")
+    count = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    for t in (5, 6):                            # the second round takes its counts from the first one's kernel
+        a = dx.host().copy()
+        want = a.copy()
+        oracle.sgd(a, g, 0.1)
+        arena.fill_(123.0)
+        sb.saps_round_pack_rows(ctx, dx.ptr, dg.ptr, 0.1, pairs, t, p, d_table, idx, count)
+        torch.cuda.synchronize()
+        assert sb.saps_status(ctx) == 0
+        m = oracle.gossip_round(want, g, 0.1, pairs, 19, t, p)
+        wv, wi, wc = oracle.pack(a, m, cap)
+        assert int(count.cpu().numpy().view(np.uint32)[0]) == wc
+        assert (idx.cpu().numpy().view(np.uint32)[:wc] == wi[:wc]).all()
+        got = arena.cpu().numpy().reshape(n, slot)
+        for i in range(n):
+            row = got[order[i]]
+            if i == skipped:
+                assert (row == 123.0).all()
+            else:
+                assert_bits_equal(row[:wc], wv[i, :wc], f"worker {i}, round {t}")
+                assert (row[wc:] == 123.0).all()
+        assert_bits_equal(dx.host(), want, "round result with per-worker destinations")
+    assert dx.canaries_intact() and dg.canaries_intact()
+    assert sb._lib.saps_round_pack_rows(ctx, dx.ptr, dg.ptr, 0.1, sb._pairs(pairs), 7, p, None, sb._ptr(idx),
+                                        sb._ptr(count), None) == sb.SAPS_ERR_INVALID
+    sb.saps_destroy(ctx)
+
+
 def test_unfused_wire_path_equals_fused_round(sb):
     # SGD-only round -> pack -> average the two packed buffers -> scatter  ==  fused round
     torch = torch_cuda()
