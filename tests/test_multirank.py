@@ -97,6 +97,41 @@ def test_plan_row_exchange_splits_a_matching():
         plan_row_exchange([1, 2, 0, 3], 0, 2, 2)
 
 
+def test_destination_table_sends_every_row_where_its_receiver_looks():
+    # Direct form: rank r's pass writes worker i's packed row to an address in the peer rank's
+    # receive buffer.  With every "address" a (rank, row) code, following the tables of all ranks
+    # must put, in row j of rank q's buffer, exactly the worker that row j's plan says it
+    # averages with (src_rows[j] == j), and nothing anywhere else.
+    from paper_2002_09692_b200.row_sharded import destination_table, plan_row_exchange
+    world, per_rank, cap = 3, 4, 10
+    rng = np.random.default_rng(11)
+    bases = [1_000_000 * (q + 1) for q in range(world)]              # fake, well separated addresses
+    for _ in range(20):
+        pairs = synth.random_perfect_matching(world * per_rank, rng)
+        plans = [plan_row_exchange(pairs, r, world, per_rank) for r in range(world)]
+        arrived = {}                                                    # (rank, row) -> sending worker
+        for r in range(world):
+            table = destination_table(plans[r], pairs, r, per_rank, bases, cap)
+            assert len(table) == per_rank
+            for i, addr in enumerate(table):
+                me = r * per_rank + i
+                if int(pairs[me]) // per_rank == r:
+                    assert addr == 0                                    # local pair: nothing to send
+                    continue
+                q, off = divmod(addr, 1_000_000)
+                q -= 1
+                assert off % (4 * cap) == 0
+                assert (q, off // (4 * cap)) not in arrived
+                arrived[(q, off // (4 * cap))] = me
+        for q in range(world):
+            for j in range(per_rank):
+                peer = int(pairs[q * per_rank + j])
+                if peer // per_rank == q:
+                    assert (q, j) not in arrived and plans[q].src_rows[j] == -1
+                else:
+                    assert arrived[(q, j)] == peer and plans[q].src_rows[j] == j
+
+
 def _row_worker(rank, world, port, results):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     dist.init_process_group("gloo", rank=rank, world_size=world)
