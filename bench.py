@@ -95,24 +95,73 @@ def measured_peak_hbm():
 
 
 class ClockSampler:
-    """nvidia-smi clock and throttle-reason samples while the timed region runs."""
+    """SM clock and throttle-reason samples while a timed region runs.
+
+    The samples come from NVML (the library behind nvidia-smi), read by a thread of this process
+    every 2 ms, so that even a region of some ten milliseconds holds several of them; where the
+    NVML binding is missing, from `nvidia-smi --query-gpu=... -lms 20` as a child process.
+    Reading clocks changes no setting of the GPU.  stop(t0, t1) keeps the samples taken between
+    the two time.perf_counter() values (those of the timed region); if the region was too short
+    to hold one, the nearest sample on either side is used and the result says so."""
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    REASON_BITS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
-    def __init__(self, gpu_id):
+    def __init__(self, gpu_id, period_s=0.002):
         """gpu_id: what `nvidia-smi -i` accepts (an index or a "GPU-<uuid>" string)."""
-        gpu_index = gpu_id
+        import threading
+        self.gpu_id = gpu_id
+        self.samples = []            # (perf_counter, sm MHz, reason names)
+        self.smax = None
+        self.source = None
+        self.proc = self.tmp = self.thread = None
+        self._stop = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            if isinstance(gpu_id, str):
+                try:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(gpu_id)
+                except Exception:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(gpu_id.encode())
+            else:
+                h = pynvml.nvmlDeviceGetHandleByIndex(int(gpu_id))
+            self.smax = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            reasons_of = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                pynvml.nvmlDeviceGetCurrentClocksThrottleReasons
+
+            def poll():
+                while not self._stop.is_set():
+                    try:
+                        mhz = float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                        mask = int(reasons_of(h))
+                    except Exception:
+                        break
+                    self.samples.append((time.perf_counter(), mhz,
+                                         tuple(name for bit, name in self.REASON_BITS.items() if mask & bit)))
+                    self._stop.wait(period_s)
+
+            poll_once = (float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)), int(reasons_of(h)))
+            del poll_once                       # both queries work on this GPU: use the thread
+            self.thread = threading.Thread(target=poll, daemon=True)
+            self.thread.start()
+            self.source = "nvml, one sample every 2 ms"
+        except Exception:
+            self._start_smi()
+
+    def _start_smi(self):
+        self.source = "nvidia-smi -lms 20"
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.proc = None
+        self.t_launch = time.perf_counter()
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "20", "-i", str(gpu_index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                 "-lms", "20", "-i", str(self.gpu_id)], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             pass
 
-    def stop(self):
+    def _collect_smi(self):
         if self.proc is not None:
             self.proc.terminate()
             try:
@@ -121,26 +170,41 @@ class ClockSampler:
                 self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
-        sm, smax, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.tmp:
             f = [v.strip() for v in line.split(",")]
             if len(f) < 9:
                 continue
             try:
-                sm.append(float(f[1]))
-                smax.append(float(f[2]))
+                mhz, smax = float(f[1]), float(f[2])
             except ValueError:
                 continue
-            for name, v in zip(names, f[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
+            self.smax = smax if self.smax is None else max(self.smax, smax)
+            # no time stamps in this mode: every sample counts as inside the window
+            self.samples.append((None, mhz, tuple(n for n, v in zip(names, f[5:9]) if v.lower().startswith("active"))))
         self.tmp.close()
         os.unlink(self.tmp.name)
-        if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
-                "samples": len(sm)}
+
+    def stop(self, t0=None, t1=None):
+        self._stop.set()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        if self.tmp is not None:
+            self._collect_smi()
+        every = list(self.samples)
+        inside = [s for s in every if s[0] is None or t0 is None or (t0 <= s[0] <= t1)]
+        note = None
+        if not inside and every:
+            mid = 0.5 * (t0 + t1)
+            inside = sorted(every, key=lambda s: abs(s[0] - mid))[:2]
+            note = "the region held no sample: the two nearest in time are given"
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "source": self.source}
+        out = {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": self.smax,
+               "reasons": sorted({r for s in inside for r in s[2]}), "samples": len(inside), "source": self.source}
+        if note:
+            out["note"] = note
+        return out
 
 
 def dist_env():
@@ -319,15 +383,17 @@ def run_ours(args):
     except Exception:
         smi_id = local
     sampler = ClockSampler(smi_id)
-    time.sleep(0.3)
+    if sampler.thread is None:
+        time.sleep(0.3)                     # a child process needs a moment before its first sample
     barrier()
+    host_t0 = time.perf_counter()
     ev_start.record(stream)
     for k in range(K):
         step(t)
         t += 1
     ev_stop.record(stream)
     barrier()
-    clocks = sampler.stop()
+    clocks = sampler.stop(host_t0, time.perf_counter())
     st = sb.saps_status(ctx)
     if st != 0:
         raise SystemExit(f"device status after the timed region: {sb.saps_strerror(st)}")
@@ -415,13 +481,15 @@ def run_ours(args):
         torch.cuda.synchronize()
         reps = int(max(20, min(5000, min_ms / max(e0.elapsed_time(e1) / 10, 1e-3))))
         sampler = ClockSampler(smi_id)
-        time.sleep(0.3)
+        if sampler.thread is None:
+            time.sleep(0.3)
+        h0 = time.perf_counter()
         e0.record(stream)
         for i in range(reps):
             fn(t + 13 + i)
         e1.record(stream)
         torch.cuda.synchronize()
-        c = sampler.stop()
+        c = sampler.stop(h0, time.perf_counter())
         return e0.elapsed_time(e1) / reps, {"sm_mhz": c["sm_mhz"], "reasons": c["reasons"], "launches": reps}
 
     pairs_fixed = sb.saps_select_peers(ctx, B, t, n)

@@ -239,8 +239,9 @@ SAPS_API int saps_unpack_avg_rows(saps_ctx* ctx, float* x, const float* recv_val
  * Instead the tile states of the compaction scan live in a fixed array inside the library
  * image (524,304 bytes).  The CUDA runtime creates that array on a GPU when it loads the
  * library's device code there (at the latest on the first launch of one of its kernels on
- * that GPU), not on demand from this call, and keeps it until the process exits.  That array covers N <= SAPS_NOALLOC_MAX_N columns; a larger context is refused
- * with SAPS_ERR_TOO_LARGE before anything is launched.
+ * that GPU), not on demand from this call, and keeps it until the process exits.  That array
+ * covers N <= SAPS_NOALLOC_MAX_N columns; a larger context is refused with SAPS_ERR_TOO_LARGE
+ * before anything is launched.
  *
  * Arguments and results are those of saps_pack (same capacity rule, same overflow
  * behaviour), plus

@@ -16,7 +16,7 @@ namespace {
 // Scratch of the allocation-free compaction entry point: the same layout as a context's
 // scratch (status word, ticket, tile states) for up to kStaticMaxTiles column
 // tiles.  Every GPU that loads the library holds these bytes until the process exits.
-__device__ __align__(256) unsigned char g_static_scratch[16 + (size_t)kStaticMaxTiles * 8];
+static __device__ __align__(256) unsigned char g_static_scratch[16 + (size_t)kStaticMaxTiles * 8];
 
 constexpr unsigned long long kFlagAggregate = 1ull << 32;
 constexpr unsigned long long kFlagInclusive = 2ull << 32;

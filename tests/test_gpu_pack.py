@@ -321,7 +321,7 @@ def test_threshold_comparison_is_strict_on_the_gpu(sb):
 
 
 @pytest.mark.parametrize("N,ld", [(70_003, 70_016), (70_003, 70_003), (70_002, 70_002)])   # 128-, 32-, 64-bit access
-@pytest.mark.parametrize("scheduler", [False, True])
+@pytest.mark.parametrize("scheduler", [False, True, "rows"])
 def test_fused_emission_overflow_is_clamped_and_reported(sb, N, ld, scheduler):
     # The count is Binomial(N, p), so a hard wire-buffer size can be exceeded (Eq. 2 / Section II-B).
     # With a capacity below the true count the emitting round must: keep the model exactly
@@ -341,7 +341,11 @@ def test_fused_emission_overflow_is_clamped_and_reported(sb, N, ld, scheduler):
     idx = torch.full((cap + guard,), -1, dtype=torch.int32, device="cuda")
     T = len(pairs_list)
     counts = torch.full((T + 1,), -1, dtype=torch.int32, device="cuda")
-    if scheduler:
+    if scheduler == "rows":                              # one destination per worker, same clamp
+        table = torch.tensor([vals.data_ptr() + 4 * cap * i for i in range(n)], dtype=torch.int64, device="cuda")
+        for r in range(T):
+            sb.saps_round_pack_rows(ctx, dx.ptr, dg.ptr, lr, pairs_list[r], 1 + r, p, table, idx, counts[r:])
+    elif scheduler:
         sb.saps_run_rounds_pack(ctx, dx.ptr, dg.ptr, lr, 1, T, p, vals, idx, counts, pairs_list=pairs_list)
     else:
         for r in range(T):
