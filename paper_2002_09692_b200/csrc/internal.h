@@ -74,6 +74,7 @@ struct RoundArgs {
     int gossip_first;      // 0: Algorithm 2's order (SGD, then average); 1: Eq. 7's order
     int staging;           // 0: chosen by size; 1: loads and stores from registers; 2: bulk copies through shared memory
     int staging_give_up;   // test hook: the staged form treats its wait for the copies as run out
+    int store_all;         // round without gradient: write unchanged vectors too (dense masks)
     // emission of the wire buffer (all NULL/0 when not emitting).  The ranks of a tile's kept
     // columns start at the number of kept columns in all earlier tiles.  That number is summed by
     // the block itself from two small arrays: the kept columns per tile, and their sums over

@@ -397,7 +397,10 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
                         *reinterpret_cast<float4*>(&s_stage[0][v]) = make_float4(va[u].v[0], va[u].v[1], va[u].v[2], va[u].v[3]);
                         *reinterpret_cast<float4*>(&s_stage[2][v]) = make_float4(vb[u].v[0], vb[u].v[1], vb[u].v[2], vb[u].v[3]);
                     }
-                } else if (HAS_G || bits[u]) {
+                } else if (HAS_G || a.store_all || bits[u]) {
+                    // without a gradient only vectors with a kept column change; for dense masks
+                    // (store_all) whole rows are written all the same, because many scattered
+                    // 16-byte stores cost more than one coalesced stream of unchanged values
                     store_stream<VEC>(xa + col[u], va[u]);
                     store_stream<VEC>(xb + col[u], vb[u]);
                 }

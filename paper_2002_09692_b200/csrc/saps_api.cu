@@ -161,6 +161,9 @@ RoundArgs round_args(const saps_ctx* ctx, float* x, const float* g, float lr, co
     a.gossip_first = ctx->gossip_first;
     a.staging = ctx->staging;
     a.staging_give_up = ctx->staging_give_up;
+    // a round without gradient rewrites only the vectors that hold a kept column, unless the mask
+    // is so dense (more than one column in 25) that a full coalesced write stream is cheaper
+    a.store_all = key.all || key.thr32 > 0x0A3D70A3u;
     a.out_vals = nullptr;
     a.out_rows = nullptr;
     a.cap = 0;
