@@ -64,7 +64,7 @@ extern "C" {
 #define SAPS_ERR_PAIRS    (-2)  /* pairs is not an involution on 0..n-1                    */
 #define SAPS_ERR_CUDA     (-3)  /* a CUDA runtime call failed (no device, launch error)    */
 #define SAPS_ERR_OVERFLOW (-4)  /* more kept columns than the pack capacity (device-found) */
-#define SAPS_ERR_TIMEOUT  (-5)  /* the compaction scan gave up waiting (device-found)      */
+#define SAPS_ERR_TIMEOUT  (-5)  /* a bounded device-side wait ran out (device-found)       */
 #define SAPS_ERR_NOMEM    (-6)  /* host or device allocation failed                        */
 #define SAPS_ERR_TOO_LARGE (-7) /* N beyond the static scratch of saps_pack_noalloc        */
 

@@ -945,7 +945,7 @@ const char* saps_strerror(int status)
         case SAPS_ERR_PAIRS: return "pairs is not an involution on 0..n-1";
         case SAPS_ERR_CUDA: return "CUDA runtime call failed";
         case SAPS_ERR_OVERFLOW: return "more kept columns than the pack capacity";
-        case SAPS_ERR_TIMEOUT: return "compaction scan gave up waiting for a predecessor tile";
+        case SAPS_ERR_TIMEOUT: return "a bounded wait on the device ran out (compaction look-back or staged copies)";
         case SAPS_ERR_NOMEM: return "out of memory";
         case SAPS_ERR_TOO_LARGE: return "N exceeds what the static scratch area of saps_pack_noalloc covers";
         default: return "unknown status";
