@@ -75,6 +75,7 @@ struct RoundArgs {
     int staging;           // 0: chosen by size; 1: loads and stores from registers; 2: bulk copies through shared memory
     int staging_give_up;   // test hook: the staged form treats its wait for the copies as run out
     int store_all;         // round without gradient: write unchanged vectors too (dense masks)
+    int store_sectors;     // round without gradient: rows start on 32-byte boundaries, store whole sectors
     // emission of the wire buffer (all NULL/0 when not emitting).  The ranks of a tile's kept
     // columns start at the number of kept columns in all earlier tiles.  That number is summed by
     // the block itself from two small arrays: the kept columns per tile, and their sums over

@@ -370,6 +370,22 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
         }
     }
 
+    // Without a gradient only vectors that hold a kept column change, so only those are stored.
+    // Where every row starts on a 32-byte boundary (store_sectors), the threads that share a
+    // 32-byte sector store together when any of them has a kept column: DRAM then receives whole
+    // sectors and never has to merge a partial one with what it holds.
+    uint32_t rewrite[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        rewrite[u] = bits[u];
+        if constexpr (!HAS_G && VEC < 8) {
+            if (a.store_sectors) {
+#pragma unroll
+                for (int d = 1; d < 8 / VEC; d <<= 1) rewrite[u] |= __shfl_xor_sync(0xFFFFFFFFu, rewrite[u], d);
+            }
+        }
+    }
+
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         if (inb[u]) {
@@ -397,10 +413,9 @@ __global__ void __launch_bounds__(kThreads, VEC == 4 ? 5 : 1) round_kernel(const
                         *reinterpret_cast<float4*>(&s_stage[0][v]) = make_float4(va[u].v[0], va[u].v[1], va[u].v[2], va[u].v[3]);
                         *reinterpret_cast<float4*>(&s_stage[2][v]) = make_float4(vb[u].v[0], vb[u].v[1], vb[u].v[2], vb[u].v[3]);
                     }
-                } else if (HAS_G || a.store_all || bits[u]) {
-                    // without a gradient only vectors with a kept column change; for dense masks
-                    // (store_all) whole rows are written all the same, because many scattered
-                    // 16-byte stores cost more than one coalesced stream of unchanged values
+                } else if (HAS_G || a.store_all || rewrite[u]) {
+                    // for dense masks (store_all) whole rows are written all the same, because many
+                    // scattered stores cost more than one coalesced stream of unchanged values
                     store_stream<VEC>(xa + col[u], va[u]);
                     store_stream<VEC>(xb + col[u], vb[u]);
                 }

@@ -164,6 +164,7 @@ RoundArgs round_args(const saps_ctx* ctx, float* x, const float* g, float lr, co
     // a round without gradient rewrites only the vectors that hold a kept column, unless the mask
     // is so dense (more than one column in 25) that a full coalesced write stream is cheaper
     a.store_all = key.all || key.thr32 > 0x0A3D70A3u;
+    a.store_sectors = reinterpret_cast<uintptr_t>(x) % 32 == 0 && (a.ld * sizeof(float)) % 32 == 0;
     a.out_vals = nullptr;
     a.out_rows = nullptr;
     a.cap = 0;
