@@ -163,6 +163,16 @@ struct SelectState {
     int t_thres = 0;  // 0 = default
     uint64_t last_t = 0;
     std::vector<int64_t> R;  // n x n, kNever = never
+    // what the last call derived from its bandwidth matrix, reused while the caller keeps passing
+    // the same matrix and threshold setting (the usual case: one matrix for a whole run)
+    std::vector<double> seen_bandwidth;   // the matrix as it was passed in
+    std::vector<double> sym_bandwidth;    // min(B, B^T), zero diagonal
+    double seen_b_thres_setting = 0.0;
+    bool seen_b_thres_default = false;
+    double derived_b_thres = 0.0;
+    uint64_t any_link[kMaxWorkers] = {};    // row masks: links with B_ij > 0
+    uint64_t fast_link[kMaxWorkers] = {};   // row masks: links of B* (B_ij >= B_thres)
+    bool derived_valid = false;
 };
 
 constexpr int64_t kNever = -(1LL << 62);

@@ -19,25 +19,30 @@ namespace saps {
 namespace {
 
 // Maximum-cardinality matching in a general graph: breadth-first alternating trees with
-// blossoms kept contracted through a "base" label per vertex.
+// blossoms kept contracted through a "base" label per vertex.  n <= 64: a row of the adjacency
+// matrix is one 64-bit mask (bit w of row v = edge v-w), neighbours are visited in ascending order
+// by peeling the lowest set bit, and all working storage is fixed-size.
 class BlossomMatcher {
 public:
-    BlossomMatcher(int n, const std::vector<uint8_t>& adj)
-        : n_(n), adj_(adj), mate_(n, -1), up_(n), base_(n), seen_(n), in_blossom_(n), on_path_(n), fifo_(n) {}
+    BlossomMatcher(int n, const uint64_t* rows) : n_(n), row_(rows)
+    {
+        for (int v = 0; v < n; ++v) mate_[v] = -1;
+    }
 
-    const std::vector<int>& solve()
+    const int* solve()
     {
         // start from a greedy matching (first free neighbour of every free vertex): on the dense
         // graphs of this rule it is already close to maximum, and only the few vertices it
         // leaves free need a search for an augmenting path
+        uint64_t free_mask = n_ == 64 ? ~0ull : ((1ull << n_) - 1);
         for (int v = 0; v < n_; ++v) {
             if (mate_[v] != -1) continue;
-            for (int w = 0; w < n_; ++w) {
-                if (w != v && mate_[w] == -1 && edge(v, w)) {
-                    mate_[v] = w;
-                    mate_[w] = v;
-                    break;
-                }
+            const uint64_t cand = row_[v] & free_mask & ~(1ull << v);
+            if (cand != 0) {
+                const int w = __builtin_ctzll(cand);
+                mate_[v] = w;
+                mate_[w] = v;
+                free_mask &= ~((1ull << v) | (1ull << w));
             }
         }
         for (int v = 0; v < n_; ++v) {
@@ -56,32 +61,30 @@ public:
     }
 
 private:
-    bool edge(int a, int b) const { return adj_[(size_t)a * n_ + b] != 0; }
-
     // first common blossom base on the two root paths
     int common_base(int a, int b)
     {
-        std::fill(on_path_.begin(), on_path_.end(), 0);
+        uint64_t on_path = 0;
         for (int v = a;;) {
             v = base_[v];
-            on_path_[v] = 1;
+            on_path |= 1ull << v;
             if (mate_[v] == -1) break;
             v = up_[mate_[v]];
         }
         for (int v = b;;) {
             v = base_[v];
-            if (on_path_[v]) return v;
+            if ((on_path >> v) & 1ull) return v;
             v = up_[mate_[v]];
         }
     }
 
     // walk from v down to the blossom base b, marking the bases on the way and re-hanging
     // the odd vertices so that the path can later be flipped in either direction
-    void mark_side(int v, int b, int child)
+    void mark_side(int v, int b, int child, uint64_t& in_blossom)
     {
         while (base_[v] != b) {
-            in_blossom_[base_[v]] = 1;
-            in_blossom_[base_[mate_[v]]] = 1;
+            in_blossom |= 1ull << base_[v];
+            in_blossom |= 1ull << base_[mate_[v]];
             up_[v] = child;
             child = mate_[v];
             v = up_[mate_[v]];
@@ -91,34 +94,36 @@ private:
     // returns the free vertex that ends an augmenting path from root, or -1
     int grow_tree(int root)
     {
-        std::fill(seen_.begin(), seen_.end(), 0);
-        std::fill(up_.begin(), up_.end(), -1);
-        for (int i = 0; i < n_; ++i) base_[i] = i;
+        uint64_t seen = 1ull << root;
+        for (int i = 0; i < n_; ++i) {
+            up_[i] = -1;
+            base_[i] = i;
+        }
         int head = 0, tail = 0;
         fifo_[tail++] = root;
-        seen_[root] = 1;
         while (head < tail) {
             const int v = fifo_[head++];
-            for (int w = 0; w < n_; ++w) {
-                if (!edge(v, w) || base_[v] == base_[w] || mate_[v] == w) continue;
+            for (uint64_t nb = row_[v]; nb != 0; nb &= nb - 1) {
+                const int w = __builtin_ctzll(nb);
+                if (base_[v] == base_[w] || mate_[v] == w) continue;
                 if (w == root || (mate_[w] != -1 && up_[mate_[w]] != -1)) {
                     // w is an even vertex of the tree: odd cycle, contract it
                     const int b = common_base(v, w);
-                    std::fill(in_blossom_.begin(), in_blossom_.end(), 0);
-                    mark_side(v, b, w);
-                    mark_side(w, b, v);
+                    uint64_t in_blossom = 0;
+                    mark_side(v, b, w, in_blossom);
+                    mark_side(w, b, v, in_blossom);
                     for (int i = 0; i < n_; ++i) {
-                        if (!in_blossom_[base_[i]]) continue;
+                        if (!((in_blossom >> base_[i]) & 1ull)) continue;
                         base_[i] = b;
-                        if (!seen_[i]) {
-                            seen_[i] = 1;
+                        if (!((seen >> i) & 1ull)) {
+                            seen |= 1ull << i;
                             fifo_[tail++] = i;
                         }
                     }
                 } else if (up_[w] == -1) {
                     up_[w] = v;
                     if (mate_[w] == -1) return w;
-                    seen_[mate_[w]] = 1;
+                    seen |= 1ull << mate_[w];
                     fifo_[tail++] = mate_[w];
                 }
             }
@@ -127,16 +132,23 @@ private:
     }
 
     int n_;
-    const std::vector<uint8_t>& adj_;
-    std::vector<int> mate_, up_, base_;
-    std::vector<char> seen_, in_blossom_, on_path_;
-    std::vector<int> fifo_;
+    const uint64_t* row_;
+    int mate_[kMaxWorkers], up_[kMaxWorkers], base_[kMaxWorkers], fifo_[kMaxWorkers];
 };
 
+// Adjacency rows (bit j of row i) of a 0/1 matrix stored as bytes.
+void rows_of(int n, const std::vector<uint8_t>& E, uint64_t* rows)
+{
+    for (int i = 0; i < n; ++i) {
+        uint64_t bits = 0;
+        for (int j = 0; j < n; ++j) bits |= (uint64_t)(E[(size_t)i * n + j] != 0 && i != j) << j;
+        rows[i] = bits;
+    }
+}
+
 // RandomlyMaxMatch: relabel the vertices by a keyed shuffle, match, map back.
-// Returns the number of matched pairs; mate[v] = partner or -1.
-int randomly_max_match(int n, const std::vector<uint8_t>& E, uint64_t seed, uint64_t t, uint32_t stage,
-                       std::vector<int>& mate)
+// rows: adjacency of E as 64-bit masks.  Returns the number of matched pairs; mate[v] = partner or -1.
+int randomly_max_match(int n, const uint64_t* rows, uint64_t seed, uint64_t t, uint32_t stage, int* mate)
 {
     const uint64_t s = seed ^ 0x5350454552ull;
     uint32_t h = mix32((uint32_t)(s & 0xFFFFFFFFull) ^ kSeedPad);
@@ -144,19 +156,24 @@ int randomly_max_match(int n, const std::vector<uint8_t>& E, uint64_t seed, uint
     h = mix32(h ^ (uint32_t)(t & 0xFFFFFFFFull));
     h = mix32(h ^ (uint32_t)(t >> 32));
     h = mix32(h ^ stage);
-    std::vector<int> perm(n);
+    int perm[kMaxWorkers], where[kMaxWorkers];
     for (int i = 0; i < n; ++i) perm[i] = i;
     for (int j = n - 1; j >= 1; --j) {
         const uint32_t r = mix32(h ^ (uint32_t)j) % (uint32_t)(j + 1);
         std::swap(perm[j], perm[r]);
     }
-    std::vector<uint8_t> P((size_t)n * n);
-    for (int a = 0; a < n; ++a)
-        for (int b = 0; b < n; ++b) P[(size_t)a * n + b] = E[(size_t)perm[a] * n + perm[b]];
+    for (int a = 0; a < n; ++a) where[perm[a]] = a;
+    // relabelled graph: vertex a stands for perm[a]; its neighbours are where[] of perm[a]'s
+    uint64_t P[kMaxWorkers];
+    for (int a = 0; a < n; ++a) {
+        uint64_t bits = 0;
+        for (uint64_t m = rows[perm[a]]; m != 0; m &= m - 1) bits |= 1ull << where[__builtin_ctzll(m)];
+        P[a] = bits;
+    }
     BlossomMatcher m(n, P);
-    const std::vector<int>& pm = m.solve();
-    mate.assign(n, -1);
+    const int* pm = m.solve();
     int pairs = 0;
+    for (int i = 0; i < n; ++i) mate[i] = -1;
     for (int a = 0; a < n; ++a) {
         if (pm[a] != -1) {
             mate[perm[a]] = perm[pm[a]];
@@ -168,8 +185,10 @@ int randomly_max_match(int n, const std::vector<uint8_t>& E, uint64_t seed, uint
 
 int matching_size(int n, const std::vector<uint8_t>& E)
 {
-    BlossomMatcher m(n, E);
-    const std::vector<int>& mate = m.solve();
+    uint64_t rows[kMaxWorkers];
+    rows_of(n, E, rows);
+    BlossomMatcher m(n, rows);
+    const int* mate = m.solve();
     int pairs = 0;
     for (int v = 0; v < n; ++v) pairs += mate[v] > v;
     return pairs;
@@ -239,33 +258,61 @@ int select_peers(SelectState& st, const double* bandwidth, uint64_t t, int32_t* 
 {
     const int n = st.n;
     if (t < st.last_t) return SAPS_ERR_INVALID;
-    for (int i = 0; i < n * n; ++i)
-        if (bandwidth[i] != bandwidth[i] || bandwidth[i] < 0.0) return SAPS_ERR_INVALID;
+    // Everything that depends on the bandwidth matrix and the threshold setting alone is derived
+    // once and kept while the caller passes the same values again (compared byte for byte).
+    const size_t cells = (size_t)n * n;
+    const bool same_setting = st.seen_b_thres_default == st.b_thres_default &&
+                              (st.b_thres_default || std::memcmp(&st.seen_b_thres_setting, &st.b_thres, sizeof(double)) == 0);
+    if (!(st.derived_valid && same_setting && st.seen_bandwidth.size() == cells &&
+          std::memcmp(st.seen_bandwidth.data(), bandwidth, cells * sizeof(double)) == 0)) {
+        st.derived_valid = false;
+        for (size_t i = 0; i < cells; ++i)
+            if (bandwidth[i] != bandwidth[i] || bandwidth[i] < 0.0) return SAPS_ERR_INVALID;
 
-    // B_ij = B_ji = min(B_ij, B_ji)
-    std::vector<double> B((size_t)n * n, 0.0);
-    for (int i = 0; i < n; ++i)
-        for (int j = 0; j < n; ++j)
-            if (i != j) B[(size_t)i * n + j] = std::min(bandwidth[(size_t)i * n + j], bandwidth[(size_t)j * n + i]);
-
-    double b_thres = st.b_thres;
-    if (std::isinf(b_thres) && b_thres > 0.0) {
-        b_thres = bottleneck_threshold(n, B);
-    } else if (st.b_thres_default) {
-        std::vector<double> links;
-        links.reserve((size_t)n * (n - 1) / 2);
+        // B_ij = B_ji = min(B_ij, B_ji)
+        std::vector<double>& S = st.sym_bandwidth;
+        S.assign(cells, 0.0);
         for (int i = 0; i < n; ++i)
-            for (int j = i + 1; j < n; ++j) links.push_back(B[(size_t)i * n + j]);
-        // median without a full sort: the upper middle element, then the largest below it
-        const size_t m = links.size();
-        if (m == 0) {
-            b_thres = 0.0;
-        } else {
-            std::nth_element(links.begin(), links.begin() + m / 2, links.end());
-            const double upper = links[m / 2];
-            b_thres = m % 2 ? upper : 0.5 * (*std::max_element(links.begin(), links.begin() + m / 2) + upper);
+            for (int j = 0; j < n; ++j)
+                if (i != j) S[(size_t)i * n + j] = std::min(bandwidth[(size_t)i * n + j], bandwidth[(size_t)j * n + i]);
+
+        double thres = st.b_thres;
+        if (std::isinf(thres) && thres > 0.0) {
+            thres = bottleneck_threshold(n, S);
+        } else if (st.b_thres_default) {
+            std::vector<double> links;
+            links.reserve((size_t)n * (n - 1) / 2);
+            for (int i = 0; i < n; ++i)
+                for (int j = i + 1; j < n; ++j) links.push_back(S[(size_t)i * n + j]);
+            // median without a full sort: the upper middle element, then the largest below it
+            const size_t m = links.size();
+            if (m == 0) {
+                thres = 0.0;
+            } else {
+                std::nth_element(links.begin(), links.begin() + m / 2, links.end());
+                const double upper = links[m / 2];
+                thres = m % 2 ? upper : 0.5 * (*std::max_element(links.begin(), links.begin() + m / 2) + upper);
+            }
         }
+        // links with B_ij > 0 and links of B* as row masks
+        for (int i = 0; i < n; ++i) {
+            uint64_t any = 0, fast = 0;
+            const double* b = &S[(size_t)i * n];
+            for (int j = 0; j < n; ++j) {
+                any |= (uint64_t)(b[j] > 0.0) << j;
+                fast |= (uint64_t)(b[j] > 0.0 && b[j] >= thres) << j;
+            }
+            st.any_link[i] = any & ~(1ull << i);
+            st.fast_link[i] = fast & ~(1ull << i);
+        }
+        st.seen_bandwidth.assign(bandwidth, bandwidth + cells);
+        st.seen_b_thres_setting = st.b_thres;
+        st.seen_b_thres_default = st.b_thres_default;
+        st.derived_b_thres = thres;
+        st.derived_valid = true;
     }
+    const uint64_t* any_link = st.any_link;
+    const uint64_t* fast_link = st.fast_link;
     int t_thres = st.t_thres;
     if (t_thres == 0) {
         int lg = 0;
@@ -288,25 +335,24 @@ int select_peers(SelectState& st, const double* bandwidth, uint64_t t, int32_t* 
     std::vector<int> label;
     const int ncomp = label_components(n, Q, label);
 
-    std::vector<uint8_t> E((size_t)n * n, 0);
-    for (int i = 0; i < n; ++i)
-        for (int j = 0; j < n; ++j) {
-            if (i == j) continue;
-            const double b = B[(size_t)i * n + j];
-            E[(size_t)i * n + j] = ncomp == 1 ? (b >= b_thres && b > 0.0)        // E = B*
-                                              : (label[i] != label[j] && b > 0.0);  // GetOverTimeMatrix
-        }
+    uint64_t E[kMaxWorkers] = {};
+    if (ncomp == 1) {
+        for (int i = 0; i < n; ++i) E[i] = fast_link[i];                      // E = B*
+    } else {
+        uint64_t members[kMaxWorkers] = {};                                    // GetOverTimeMatrix
+        for (int i = 0; i < n; ++i) members[label[i]] |= 1ull << i;
+        for (int i = 0; i < n; ++i) E[i] = any_link[i] & ~members[label[i]];
+    }
 
-    std::vector<int> mate;
+    int mate[kMaxWorkers];
     const int first = randomly_max_match(n, E, st.seed, t, 1, mate);
     if (2 * first != n) {
         // GetUnmatch: every link between two still unmatched workers, bandwidth ignored
-        std::vector<uint8_t> E2((size_t)n * n, 0);
-        for (int i = 0; i < n; ++i)
-            for (int j = 0; j < n; ++j)
-                if (i != j && mate[i] == -1 && mate[j] == -1 && B[(size_t)i * n + j] > 0.0)
-                    E2[(size_t)i * n + j] = 1;
-        std::vector<int> mate2;
+        uint64_t unmatched = 0;
+        for (int i = 0; i < n; ++i) unmatched |= (uint64_t)(mate[i] == -1) << i;
+        uint64_t E2[kMaxWorkers] = {};
+        for (int i = 0; i < n; ++i) E2[i] = ((unmatched >> i) & 1ull) ? (any_link[i] & unmatched) : 0ull;
+        int mate2[kMaxWorkers];
         randomly_max_match(n, E2, st.seed, t, 2, mate2);
         for (int i = 0; i < n; ++i)
             if (mate2[i] != -1) mate[i] = mate2[i];

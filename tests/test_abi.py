@@ -302,6 +302,38 @@ def test_select_peers_is_a_pure_function_of_seed_t_and_state():
         sb.saps_destroy(h)
 
 
+def test_select_peers_remembers_nothing_wrong_about_an_earlier_matrix():
+    # The library keeps what it derived from the last bandwidth matrix (symmetrised links,
+    # threshold, link masks) for as long as the caller passes the same matrix and threshold
+    # setting.  A context that sees the matrices and settings change from call to call must
+    # choose exactly what contexts do that never saw another matrix (same seed, same R history).
+    n = 16
+    mats = [synth.bandwidth_matrix(n, 1.0, 100.0, seed=s) for s in (1, 2, 3)]
+    mats[2][4, 9] = 0.0                                   # an asymmetric, partly missing link
+    settings = [(float("nan"), 0), (40.0, 0), (float("inf"), 0)]
+    mixed = sb.saps_create(n, 8, 5)
+    for t in range(1, 61):
+        B = mats[(t * 7) % 3]
+        b_thres, t_thres = settings[(t // 3) % 3]
+        # control: a fresh context brought to the same state, which has never derived anything
+        R, last = sb.saps_get_select_state(mixed, n)
+        fresh = sb.saps_create(n, 8, 5)
+        sb.saps_set_select_state(fresh, R, last)
+        sb.saps_set_select_params(fresh, b_thres, t_thres)
+        sb.saps_set_select_params(mixed, b_thres, t_thres)
+        want = sb.saps_select_peers(fresh, B, t, n)
+        got = sb.saps_select_peers(mixed, B.copy(), t, n)  # another buffer with the same values
+        assert got == want, t
+        sb.saps_destroy(fresh)
+    # an edit in place of the caller's buffer is seen
+    B = mats[0].copy()
+    sb.saps_set_select_params(mixed, 50.0, 0)
+    sb.saps_select_peers(mixed, B, 61, n)
+    B[:, :] = 0.0
+    assert sb.saps_select_peers(mixed, B, 62, n) == list(range(n))   # no links left: nobody is paired
+    sb.saps_destroy(mixed)
+
+
 def test_select_peers_odd_n_missing_links_and_bad_input():
     ctx = sb.saps_create(5, 8, 0)
     B = synth.bandwidth_matrix(5, 1.0, 100.0, seed=4)
