@@ -142,8 +142,8 @@ class ClockSampler:
                                          tuple(name for bit, name in self.REASON_BITS.items() if mask & bit)))
                     self._stop.wait(period_s)
 
-            poll_once = (float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)), int(reasons_of(h)))
-            del poll_once                       # both queries work on this GPU: use the thread
+            pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)   # both queries must work on this GPU,
+            reasons_of(h)                                            # else the except below falls back
             self.thread = threading.Thread(target=poll, daemon=True)
             self.thread.start()
             self.source = "nvml, one sample every 2 ms"
