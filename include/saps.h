@@ -43,6 +43,12 @@
  *     saps_mask, saps_unpack_avg* and saps_pack_noalloc allocate nothing.
  *   - Calls on one context must not overlap on the GPU (use one stream, or order streams
  *     with events): they share the scratch area.
+ *   - Ordinary stream order is all a caller needs: work enqueued behind a call sees its results.
+ *     One special case: the round kernels let a kernel that is launched behind them WITH the
+ *     programmatic-stream-serialization launch attribute start early (consecutive rounds overlap
+ *     at their edges that way).  A caller who launches own kernels with that attribute directly
+ *     behind a round must, as always with that attribute, call cudaGridDependencySynchronize()
+ *     in them before touching x or the wire buffers.  Kernels launched without it are unaffected.
  */
 #ifndef SAPS_H_
 #define SAPS_H_
